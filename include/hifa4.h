@@ -1,0 +1,187 @@
+/*
+ * hifa4.h -- C ABI of the HiFA4 hot path for NVIDIA B200 (sm_100a).
+ *
+ * HiFA4 (arxiv 2607.04302) runs both attention GEMMs, Q K^T and P V, on HIF4
+ * 4-bit block-floating-point values, keeps the online-softmax state in FP16,
+ * rescales post-RoPE Q and K per channel by calibration-static Smooth-QK
+ * factors, and takes the softmax normalizer from the quantized P-hat that
+ * feeds the PV GEMM (P-Reordering), produced in the same tensor-core pass by a
+ * column of ones appended to V (Algorithm 1 "C4V16-Aux").
+ *
+ * Conventions for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller unless a
+ *     parameter says "host".  The library allocates no device memory, frees
+ *     none and never synchronizes; work is enqueued on `stream`
+ *     (a cudaStream_t passed as void*; NULL is the default stream).
+ *   - Tensors are contiguous, row-major, in the index order given.
+ *   - Return value: a hifa4_status.  No exception crosses this boundary and
+ *     there is no CPU fallback: on a device that is not sm_100 every compute
+ *     call returns HIFA4_ERR_ARCH.
+ *   - `d_status` (optional, may be NULL) is a device int the kernels write a
+ *     non-zero hifa4_status into when a bounded wait inside a kernel expires;
+ *     the caller zeroes it and reads it after synchronizing.
+ */
+#ifndef HIFA4_H
+#define HIFA4_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HIFA4_OK = 0,
+    HIFA4_ERR_INVALID_ARG = 1,   /* null pointer, non-positive size, bad enum          */
+    HIFA4_ERR_UNSUPPORTED = 2,   /* shape / flag combination not built                 */
+    HIFA4_ERR_WORKSPACE = 3,     /* workspace missing or too small                     */
+    HIFA4_ERR_ARCH = 4,          /* current device is not compute capability 10.x      */
+    HIFA4_ERR_CUDA = 5,          /* a CUDA runtime/driver call failed                  */
+    HIFA4_ERR_TIMEOUT = 6        /* a bounded device-side wait expired (see d_status)  */
+} hifa4_status;
+
+typedef enum { HIFA4_F16 = 0, HIFA4_BF16 = 1, HIFA4_F32 = 2 } hifa4_dtype;
+
+enum { HIFA4_Q = 0, HIFA4_K = 1, HIFA4_V = 2 };               /* `which` */
+enum { HIFA4_PART_CODES = 0, HIFA4_PART_META = 1, HIFA4_PART_MMA = 2 }; /* `part` */
+enum { HIFA4_MAX_HEADS = 256, HIFA4_MAX_DEBUG_BLOCKS = 16 };
+
+/* Problem shape.  Q is [B,Hq,N,d]; K and V are [B,Hkv,N,d] ("GQA and batch
+ * handling", Appendix "Implementation Details").  d in {64,128,256};
+ * N a multiple of 64; Hq, Hkv <= HIFA4_MAX_HEADS.  q_to_kv is a HOST array of
+ * Hq KV-head indices, or NULL for the usual grouping h / (Hq/Hkv) (then Hq
+ * must be a multiple of Hkv).  in_dtype is HIFA4_F16 or HIFA4_BF16. */
+typedef struct {
+    int B, Hq, Hkv, N, d;
+    const int* q_to_kv;
+    int in_dtype;
+} hifa4_shape;
+
+/* Quantized Q/K/V (Algorithm 1 line 3).  Nine device buffers the caller
+ * allocates with the sizes hifa4_quant_bytes() returns.
+ *   *_codes : HIF4 element nibbles, two per byte, even element in the low
+ *             nibble; nibble = sign<<3 | m, magnitude m/4 (S1P2).
+ *   *_meta  : one uint32 per 64-element group: byte 0 the E6M2 level-1 scale
+ *             code (S = 2^(e-48) (1+M/4), e = code>>2, M = code&3), byte 1
+ *             the 8 level-2 bits (bit u covers elements 8u..8u+7), bytes 2-3
+ *             the 16 level-3 bits (bit t covers elements 4t..4t+3).
+ *             value_i = +-S * 2^(l2+l3) * m_i / 4      (Background, "HIF4").
+ *   *_mma   : the same values, dequantized exactly to BF16 (every HIF4 value
+ *             has at most 6 significant bits), in the layout the attention
+ *             kernel's TMA loads expect.
+ * Groups run along each GEMM's contraction axis: along d for Q and K
+ * (codes [B,H,N,d/2], meta [B,H,N,d/64], mma [B,H,N,d]); along tokens for V
+ * (codes [B,Hkv,d,N/2], meta [B,Hkv,d,N/64], mma [B,Hkv,d,N], i.e. V is
+ * stored transposed). */
+typedef struct {
+    uint8_t* q_codes; uint32_t* q_meta; void* q_mma;
+    uint8_t* k_codes; uint32_t* k_meta; void* k_mma;
+    uint8_t* v_codes; uint32_t* v_meta; void* v_mma;
+} hifa4_qkv;
+
+/* Calibration result summary (host memory).  rho_K and T_KQ are the gate
+ * statistics of "Adaptive Applicability Gate"; they are NaN unless mode 3 is
+ * built.  branch: 0 bypass, 1 strong, 2 mild, 4 caller's alpha. */
+typedef struct { float rho_K, T_KQ; int branch; float alpha; } hifa4_calib_stats;
+
+/* Attention parameters.
+ *   causal      1: key j contributes to row i only if j <= i.
+ *   Br          query rows per CTA; scheduling only, must be 128.
+ *   Bc          key-tile width of the online softmax (64 or 128).  It is part
+ *               of the result: P is quantized under the running maximum that
+ *               holds after each Bc keys (Algorithm 1 lines 7-10).
+ *   normalizer  0: consistent (P-Reordering, normalizer = rowsum of P-hat via
+ *               the ones column); 1 (mismatched) is not built.
+ *   qmean       must be 0 (Q-Mean auxiliary, Algorithm 1 lines 2 and 6, not built).
+ *   p_dtype     HIFA4_F16: exp(S-m) is rounded to FP16 before quantization
+ *               ("FP16 operations", Appendix "Implementation Details").
+ *   out_dtype   HIFA4_F16 / HIFA4_BF16 / HIFA4_F32 element type of `out`.
+ *   softmax_scale  0 selects 1/sqrt(d). */
+typedef struct {
+    int causal, Br, Bc;
+    int normalizer, qmean, p_dtype, out_dtype;
+    float softmax_scale;
+} hifa4_attn_params;
+
+/* Optional debug dump of P-hat for up to HIFA4_MAX_DEBUG_BLOCKS 128-row query
+ * blocks.  blocks: HOST array of n_blocks triples (b, h, query_block_index).
+ * p_codes: device [n_blocks][128][N] bytes, the nibble of every P-hat element
+ * (0 where the key tile was skipped by causality); p_step: device
+ * [n_blocks][128][N/4] floats, the step of every 4-key subgroup; l_out, m_out:
+ * device [n_blocks][128] floats, the accumulated normalizer and the final
+ * running maximum.  Any of the four device pointers may be NULL. */
+typedef struct {
+    int n_blocks;
+    const int* blocks;
+    uint8_t* p_codes;
+    float* p_step;
+    float* l_out;
+    float* m_out;
+} hifa4_debug;
+
+const char* hifa4_status_string(int status);
+
+/* Calls made so far in this process: out[0] calibrate, out[1] quantize,
+ * out[2] attention, out[3] kernels launched (all entry points). */
+void hifa4_get_counters(unsigned long long out[4]);
+
+/* Offline Smooth-QK calibration (Eq. "sqk"; "Calibration-Static Deployment").
+ *   q_cal [S,Hq,Ncal,d], k_cal [S,Hkv,Ncal,d]: post-RoPE calibration
+ *   activations of one layer, S samples of Ncal tokens, element type dt.
+ *   Per sample and channel the statistic is the largest magnitude over tokens
+ *   (for Q also over the query heads sharing the KV head); samples are
+ *   combined by root-mean-square; s = Kagg^alpha / Qagg^(1-alpha), 1 where an
+ *   aggregate is zero.  mode: 0 bypass (s = 1), 1 strong (alpha 0.5), 2 mild
+ *   (alpha 0.25), 4 caller's alpha; 3 (gate decides) returns
+ *   HIFA4_ERR_UNSUPPORTED.
+ *   Outputs (device): s, inv_s [Hkv,d] floats, inv_s = fl32(1/s).
+ *   absmax_ws: device scratch of 2*S*Hkv*d floats; the call clears it.
+ *   host_stats: optional HOST struct, filled without synchronizing. */
+int hifa4_smooth_calibrate(const void* q_cal, const void* k_cal, int S, int Hq, int Hkv,
+                           int Ncal, int d, const int* q_to_kv, int dt, int mode, float alpha,
+                           float* s, float* inv_s, float* absmax_ws,
+                           hifa4_calib_stats* host_stats, void* stream);
+
+/* Bytes of one buffer of hifa4_qkv for this shape; 0 on a bad argument. */
+size_t hifa4_quant_bytes(const hifa4_shape* shape, int which, int part);
+
+/* Smooth-QK scaling fused with HIF4 quantization (Algorithm 1 lines 1 and 3).
+ *   q~ = round_in(q * s[kv(h)]), k~ = round_in(k * inv_s[g]) with an fp32
+ *   multiply rounded to the input dtype; V is quantized as it is.
+ *   s, inv_s: [Hkv,d] floats, or both NULL for bypass.  Any of q, k, v may be
+ *   NULL to skip that tensor.  Fills the buffers of `out`. */
+int hifa4_quantize_qkv(const hifa4_shape* shape, const void* q, const void* k, const void* v,
+                       const float* s, const float* inv_s, const hifa4_qkv* out,
+                       int* d_status, void* stream);
+
+/* Workspace the attention call needs (may be 0). */
+size_t hifa4_attention_workspace_bytes(const hifa4_shape* shape, const hifa4_attn_params* prm);
+
+/* Fused prefill attention forward on quantized operands (Algorithm 1 lines
+ * 4-13): S = Q-hat K-hat^T / sqrt(d); FP16 running max and rescale;
+ * P = exp(S - m) in FP16; P-hat = HIF4(P) per row and 64 keys;
+ * [O | l] += P-hat [V-hat | 1]; out = O / l.
+ *   qkv: buffers filled by hifa4_quantize_qkv for the same shape (only the
+ *   *_mma images are read).  out: [B,Hq,N,d] of prm->out_dtype.
+ *   workspace: at least hifa4_attention_workspace_bytes() bytes (NULL if 0).
+ *   dbg: NULL, or a P-hat dump request. */
+int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv,
+                        const hifa4_attn_params* prm, void* out, void* workspace,
+                        const hifa4_debug* dbg, int* d_status, void* stream);
+
+/* Workspace for hifa4_attention_fwd_raw: all nine hifa4_qkv buffers (each
+ * rounded up to 256 bytes) plus the attention workspace. */
+size_t hifa4_attention_raw_workspace_bytes(const hifa4_shape* shape, const hifa4_attn_params* prm);
+
+/* Algorithm 1 end to end on raw post-RoPE Q/K/V: hifa4_quantize_qkv into
+ * `workspace`, then hifa4_attention_fwd.  s, inv_s as in hifa4_quantize_qkv. */
+int hifa4_attention_fwd_raw(const hifa4_shape* shape, const void* q, const void* k, const void* v,
+                            const float* s, const float* inv_s, const hifa4_attn_params* prm,
+                            void* out, void* workspace, size_t workspace_bytes,
+                            int* d_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HIFA4_H */

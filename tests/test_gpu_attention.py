@@ -1,0 +1,120 @@
+"""GPU parity of the fused attention forward against the CPU oracle (Algorithm 1), through the
+C ABI: P-hat codes/steps, normalizer and output, on small cases element by element and on sampled
+query blocks of the full-size configurations."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_04302_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def hb():
+    from paper_2607_04302_b200 import binding
+    binding.lib()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def par():
+    from tests import parity
+    return parity
+
+
+def test_tiny_config(hb, par):
+    """Configuration 1: B=1, H=1, N=128, d=128, fp16, x20 K channels, 64x64 tiles, non-causal."""
+    cfg = synth.config("C1")
+    res = par.run_case(cfg, DEV)
+    print(par.assert_within_bars(res, "C1"))
+    assert res["rows"] == 128
+
+
+SMALL = {
+    "d128-bc128-causal-gqa": synth.config("C2", N=512, Hq=4, Hkv=2, cal_samples=4, cal_tokens=128),
+    "d128-bc64-causal": synth.config("C2", N=384, Hq=2, Hkv=1, Bc=64, cal_samples=4, cal_tokens=128),
+    "d128-bc128-noncausal": synth.config("C2", N=256, Hq=2, Hkv=2, causal=False, cal_samples=4, cal_tokens=128),
+    "d128-ragged-n": synth.config("C2", N=320, Hq=2, Hkv=1, cal_samples=4, cal_tokens=128),
+    "d128-ragged-noncausal": synth.config("C3", N=192, Hq=1, Hkv=1, causal=False),
+    "d64-bc128": synth.config("C3", N=256, Hq=2, Hkv=1, d=64),
+    "d64-bc64-fp16": synth.config("C3", N=256, Hq=2, Hkv=1, d=64, Bc=64, dtype="fp16"),
+    "d256-bc64-mild": synth.config("C4", N=256, Hq=2, Hkv=1, Bc=64, cal_samples=3, cal_tokens=64),
+    "batch2": synth.config("C5", B=2, N=256, Hq=4, Hkv=2, cal_samples=2, cal_tokens=64),
+    "n64": synth.config("C3", N=64, Hq=1, Hkv=1),
+}
+
+
+@pytest.mark.parametrize("name", list(SMALL))
+def test_small_cases_elementwise(hb, par, name):
+    cfg = SMALL[name]
+    res = par.run_case(cfg, DEV)
+    print(par.assert_within_bars(res, name))
+    assert res["rows"] == cfg.B * cfg.Hq * cfg.N
+
+
+def test_output_dtypes_and_determinism(hb, par):
+    cfg = SMALL["d128-bc128-causal-gqa"]
+    q, k, v = synth.make_qkv(cfg)
+    s, inv_s = par.calibrate(cfg, DEV)
+    qkv = hb.quantize_qkv(q.to(DEV), k.to(DEV), v.to(DEV), s, inv_s)
+    o32 = hb.attention_fwd(qkv, True, Bc=128, out_dtype=hb.F32)
+    o32b = hb.attention_fwd(qkv, True, Bc=128, out_dtype=hb.F32)
+    assert torch.equal(o32, o32b)                              # no atomics: bit-identical reruns
+    o16 = hb.attention_fwd(qkv, True, Bc=128, out_dtype=hb.F16)
+    ob16 = hb.attention_fwd(qkv, True, Bc=128, out_dtype=hb.BF16)
+    assert torch.equal(o16, o32.to(torch.float16)) and torch.equal(ob16, o32.to(torch.bfloat16))
+    # Bc is part of the result; Br is not exposed beyond 128
+    o64 = hb.attention_fwd(qkv, True, Bc=64, out_dtype=hb.F32)
+    assert not torch.equal(o64, o32)
+    assert torch.isfinite(o32).all()
+
+
+def test_raw_entry_point_equals_two_step_path(hb, par):
+    cfg = SMALL["d128-bc128-causal-gqa"]
+    q, k, v = (t.to(DEV) for t in synth.make_qkv(cfg))
+    s, inv_s = par.calibrate(cfg, DEV)
+    a = hb.attention_fwd(hb.quantize_qkv(q, k, v, s, inv_s), True, Bc=128)
+    b = hb.attention_fwd_raw(q, k, v, s, inv_s, True, Bc=128)
+    assert torch.equal(a, b)
+    with pytest.raises(hb.Hifa4Error):                          # undersized workspace is refused
+        hb.attention_fwd_raw(q, k, v, s, inv_s, True, Bc=128,
+                             workspace=torch.empty(1024, dtype=torch.uint8, device=DEV))
+
+
+def test_unsupported_flags_are_refused(hb, par):
+    cfg = SMALL["n64"]
+    q, k, v = (t.to(DEV) for t in synth.make_qkv(cfg))
+    qkv = hb.quantize_qkv(q, k, v)
+    with pytest.raises(hb.Hifa4Error):
+        hb.attention_fwd(qkv, True, Bc=96)
+    with pytest.raises(hb.Hifa4Error):
+        hb.attention_fwd(qkv, True, Bc=128, Br=64)
+
+
+def _sampled_blocks(cfg, heads):
+    n_qb = cfg.N // 128
+    return [(b, h, t) for b in (0, cfg.B - 1) for h in heads for t in sorted({0, n_qb // 2, n_qb - 1})]
+
+
+@pytest.mark.parametrize("name", ["C2", "C3", "C4"])
+def test_full_size_sampled_blocks(hb, par, name):
+    """Full-size configurations in the launch configuration the benchmark times; the oracle
+    evaluates sampled rows of the first, a middle and the last query block of two heads."""
+    over = dict(Bc=64) if name == "C4" else {}
+    cfg = synth.config(name, cal_samples=4, cal_tokens=256, **over)
+    blocks = sorted(set(_sampled_blocks(cfg, (0, cfg.Hq - 1))))
+    res = par.run_case(cfg, DEV, blocks=blocks, check_quant=(name == "C2"), rows_per_block=24)
+    print(par.assert_within_bars(res, name))
+    out = res["out"]
+    assert torch.isfinite(out).all()
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_sweep_point_sampled(hb, par, causal):
+    """Configuration 5 at N = 2048 (B = 4), causal and non-causal."""
+    cfg = synth.config("C5", N=2048, causal=causal, cal_samples=2, cal_tokens=256)
+    blocks = [(0, 0, 0), (3, 31, 15), (1, 17, 7)]
+    res = par.run_case(cfg, DEV, blocks=blocks, check_quant=False, rows_per_block=16)
+    print(par.assert_within_bars(res, f"C5 N=2048 causal={causal}"))
