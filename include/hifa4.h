@@ -108,7 +108,7 @@ typedef struct {
  * blocks.  blocks: HOST array of n_blocks triples (b, h, query_block_index).
  * p_codes: device [n_blocks][128][N] bytes, the nibble of every P-hat element
  * (0 where the key tile was skipped by causality); p_step: device
- * [n_blocks][128][N/4] floats, the step of every 4-key subgroup; l_out, m_out:
+ * [n_blocks][128][N/4] floats, the step of every 4-key subgroup (0 for an all-zero group); l_out, m_out:
  * device [n_blocks][128] floats, the accumulated normalizer and the final
  * running maximum.  Any of the four device pointers may be NULL. */
 typedef struct {

@@ -289,7 +289,7 @@ typedef struct {
 /* q_rows [R][d] raw queries, q_pos [R] their token index, k,v [N][d] raw,
  * s/inv_s [d] or NULL (bypass).  out [R][d].  Optional dumps (NULL to skip):
  *   p_codes [R][N]  nibble of every P-hat element (0 where a key tile is skipped)
- *   p_step  [R][N/4] step of every 4-key subgroup (0 where skipped)
+ *   p_step  [R][N/4] step of every 4-key subgroup (0 where skipped or where the group is all zero)
  *   p_raw   [R][N]  P before quantization,  p_hat [R][N] dequantized P-hat
  *   m_trace [R][N/Bc] running max after each processed tile (NaN if skipped)
  *   l_out   [R]     accumulated normalizer before the final division         */
@@ -419,8 +419,9 @@ int hifa4_oracle_attention_rows(const hifa4_oracle_params* p, const float* q_row
             }
             for (int j = 0; j < w; ++j) {
                 if (p_codes) p_codes[(long)row * N + j0 + j] = nib[j];
-                if (p_step && p->quant_p && (j % 4) == 0)
-                    p_step[(long)row * (N / 4) + (j0 + j) / 4] = (float)hif4_step(pmeta[j / 64], j % 64);
+                if (p_step && p->quant_p && (j % 4) == 0)      /* an all-zero group (metadata 0) reports step 0 */
+                    p_step[(long)row * (N / 4) + (j0 + j) / 4] =
+                        pmeta[j / 64] ? (float)hif4_step(pmeta[j / 64], j % 64) : 0.0f;
                 if (p_raw) p_raw[(long)row * N + j0 + j] = P[j];
                 if (p_hat) p_hat[(long)row * N + j0 + j] = Ph[j];
             }

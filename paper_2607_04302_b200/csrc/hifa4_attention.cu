@@ -280,7 +280,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
                 }
                 uint8_t* dc = nullptr;
                 float* ds = nullptr;
-                if (dbg_slot >= 0 && row < N) {
+                if (dbg_slot >= 0 && row < N && j0 + gq * 64 < N) {
                     size_t r_idx = (size_t)dbg_slot * 128 + tid;
                     if (args.dbg.p_codes) dc = args.dbg.p_codes + r_idx * N + j0 + gq * 64;
                     if (args.dbg.p_step) ds = args.dbg.p_step + r_idx * (N / 4) + (j0 + gq * 64) / 4;
