@@ -1,0 +1,346 @@
+#!/usr/bin/env python
+"""Benchmark of the HiFA4 hot path on B200: one step = Smooth-QK + HIF4 quantization of Q/K/V
+followed by the fused 4-bit-operand attention forward (Algorithm 1) over one batch of synthetic
+prefill activations.  Prints ONE JSON line ("Measurement").
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--impl ours|reference]
+
+N > 1 is launched by torch.distributed.run, one rank per GPU; every rank processes its own copy
+of the workload (independent batches: the path has no exchange step), so scaling is weak.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_04302_b200 import synth  # noqa: E402
+
+METRIC = "4-bit attention prefill TFLOPS on 1 B200; % of dense 4-bit tensor peak"
+UNIT = "TFLOP/s"
+NOMINAL = {"fp4": 9000.0, "fp8": 4500.0, "bf16": 2250.0}      # dense TFLOP/s, context only
+
+
+def attn_flops(cfg) -> float:
+    f = 4.0 * cfg.B * cfg.Hq * cfg.N * cfg.N * cfg.d
+    return f / 2 if cfg.causal else f
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], bf16=d["bf16_tflops"], bf16_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc, self.thr = index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            return
+        self.thr = threading.Thread(target=self._read, daemon=True)
+        self.thr.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = float(r[1])
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        busy = sorted(sm)[len(sm) // 2:] if sm else []          # upper half = samples under load
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_time(cfg, q, k, v, s, inv_s, heads):
+    """Time the CPU oracle, as it stands, on whole heads of the workload (batch 0)."""
+    from oracle import hifa4_oracle as orc
+    import numpy as np
+    dt = orc.F16 if cfg.dtype == "fp16" else orc.BF16
+    idx = np.arange(cfg.N, dtype=np.int32)
+    grp = cfg.Hq // cfg.Hkv
+    t0 = time.perf_counter()
+    for h in heads:
+        g = h // grp
+        orc.attention_rows(q[0, h], idx, k[0, g], v[0, g], None if s is None else s[g],
+                           None if inv_s is None else inv_s[g], causal=cfg.causal, Bc=cfg.Bc, in_dtype=dt)
+    return time.perf_counter() - t0, orc.num_threads()
+
+
+def head_flops(cfg) -> float:
+    f = 4.0 * cfg.N * cfg.N * cfg.d
+    return f / 2 if cfg.causal else f
+
+
+def host_inputs(cfg):
+    q, k, v = synth.make_qkv(cfg)
+    return q, k, v
+
+
+def oracle_scales(cfg):
+    """Smooth-QK factors from the oracle's own calibration (used by the CPU legs only)."""
+    if cfg.smooth_mode == 0:
+        return None, None
+    from oracle import hifa4_oracle as orc
+    small = synth.config(cfg.name.split("-")[0], cal_samples=min(cfg.cal_samples, 4), cal_tokens=min(cfg.cal_tokens, 256))
+    qc, kc = synth.make_calibration(small)
+    cal = orc.smooth_calibrate(qc.float().numpy(), kc.float().numpy(), cfg.smooth_mode)
+    return cal["s"], cal["inv_s"]
+
+
+def run_reference(args, cfg, rank):
+    """--impl reference: the CPU oracle, as it stands, on a bounded sample per step."""
+    if rank != 0:
+        return
+    from oracle import hifa4_oracle as orc
+    orc.build()
+    q, k, v = (t.float().numpy() for t in host_inputs(cfg))
+    s, inv_s = oracle_scales(cfg)
+    t1, cores = oracle_time(cfg, q, k, v, s, inv_s, [0])
+    n_heads = max(1, min(cfg.Hq, int(8.0 / max(t1, 1e-3))))          # about 8 s of CPU work per step
+    heads = [int(i * cfg.Hq / n_heads) for i in range(n_heads)]
+    for _ in range(args.warmup):
+        oracle_time(cfg, q, k, v, s, inv_s, heads[:1])
+    tot = 0.0
+    for _ in range(args.steps):
+        t, cores = oracle_time(cfg, q, k, v, s, inv_s, heads)
+        tot += t
+    val = n_heads * head_flops(cfg) * args.steps / tot / 1e12
+    sample = f"{n_heads} of {cfg.B * cfg.Hq} (batch, head) slices of {cfg.name}, all {cfg.N} rows each, per step"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": cfg.name, "causal": cfg.causal, "Bc": cfg.Bc},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="C2", help="C2 (headline), C3, C4, C5 or C5@<N>")
+    ap.add_argument("--noncausal", action="store_true")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    name, _, n_over = args.workload.partition("@")
+    over = {}
+    if n_over:
+        over["N"] = int(n_over)
+    if args.noncausal:
+        over["causal"] = False
+    if name == "C4":
+        over.setdefault("Bc", 64)          # d = 256 is built with 64-key tiles
+    cfg = synth.config(name, **over)
+
+    if args.impl == "reference":
+        run_reference(args, cfg, rank)
+        return
+
+    from paper_2607_04302_b200 import binding as hb
+    hb.lib()                                  # fail loudly if the CUDA library is missing
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    # ---- inputs (resident in HBM) and offline calibration
+    big = cfg.B * cfg.Hq * cfg.N * cfg.d > (1 << 28)
+    if big:
+        q, k, v = synth.make_qkv_device(cfg, dev)
+        qh = kh = vh = None
+    else:
+        qh, kh, vh = host_inputs(cfg)
+        q, k, v = qh.to(dev), kh.to(dev), vh.to(dev)
+    s = inv_s = None
+    if cfg.smooth_mode:
+        qc, kc = synth.make_calibration(cfg, samples=min(cfg.cal_samples, 8), tokens=min(cfg.cal_tokens, 512))
+        s, inv_s = hb.smooth_calibrate(qc.to(dev), kc.to(dev), cfg.smooth_mode)
+    dt = hb._DT[q.dtype]
+    qkv = hb.alloc_qkv(cfg.B, cfg.Hq, cfg.Hkv, cfg.N, cfg.d, dt, dev)
+    out = torch.empty((cfg.B, cfg.Hq, cfg.N, cfg.d), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)       # > 126 MB of L2
+
+    def step():
+        hb.quantize_qkv(q, k, v, s, inv_s, out=qkv, d_status=status)
+        mid = torch.cuda.Event(enable_timing=True)
+        mid.record()
+        hb.attention_fwd(qkv, cfg.causal, Bc=cfg.Bc, out_dtype=hb.F32, out=out, d_status=status)
+        return mid
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        step()
+    barrier()
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    c0 = hb.get_counters()["launches"]
+    ev = []
+    barrier()
+    for _ in range(args.steps):
+        flush.zero_()                                                   # L2 flush, outside the events
+        a = torch.cuda.Event(enable_timing=True)
+        b = torch.cuda.Event(enable_timing=True)
+        a.record()
+        mid = step()
+        b.record()
+        ev.append((a, mid, b))
+    barrier()
+    launches = hb.get_counters()["launches"] - c0
+    clocks = sampler.stop()
+    step_ms = [a.elapsed_time(b) for a, _, b in ev]
+    attn_ms = [m.elapsed_time(b) for _, m, b in ev]
+    quant_ms = [a.elapsed_time(m) for a, m, _ in ev]
+    total_ms = sum(step_ms)
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+
+    # ---- end to end through the raw C-ABI entry point with host buffers (pinned), copies timed
+    e2e = None
+    if not big:
+        pq, pk, pv = qh.pin_memory(), kh.pin_memory(), vh.pin_memory()
+        po = torch.empty(out.shape, dtype=torch.float32).pin_memory()
+        dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+        ws = torch.empty(hb.attention_raw_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.N, cfg.d, dt, cfg.causal, cfg.Bc),
+                         dtype=torch.uint8, device=dev)
+
+        def e2e_step():
+            dq.copy_(pq, non_blocking=True); dk.copy_(pk, non_blocking=True); dv.copy_(pv, non_blocking=True)
+            hb.attention_fwd_raw(dq, dk, dv, s, inv_s, cfg.causal, Bc=cfg.Bc, out=out, workspace=ws, d_status=status)
+            po.copy_(out, non_blocking=True)
+
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        n_e2e = max(3, min(args.steps, 10))
+        a.record()
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record()
+        barrier()
+        e_ms = a.elapsed_time(b)
+        if dist is not None:
+            t = torch.tensor([e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        h2d = (pq.numel() + pk.numel() + pv.numel()) * pq.element_size()
+        e2e = {"value": world * attn_flops(cfg) * n_e2e / (e_ms * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": po.numel() * 4, "ms_per_step": e_ms / n_e2e}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    fl = attn_flops(cfg)
+    value = world * fl * args.steps / (total_ms * 1e-3) / 1e12
+    attn_avg_ms = sum(attn_ms) / len(attn_ms)
+    achieved = fl / (attn_avg_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "attention_fwd_kernel", "achieved": achieved, "peak": peaks["bf16"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["bf16"], "traffic": None,
+                "peak_source": f"{peaks['source']} cuBLAS bf16 burst (the MMA kind issued is kind::f16 on BF16 images)",
+                "avg_launch_ms": attn_avg_ms,
+                "frac_of_nominal": {k_: achieved / v_ for k_, v_ in NOMINAL.items()}}
+    q_bytes = sum(t.numel() for t in (q, k, v)) * (2 + 0.5625)
+    quant = {"avg_ms": sum(quant_ms) / len(quant_ms), "algorithmic_gbs": q_bytes / (sum(quant_ms) / len(quant_ms) * 1e-3) / 1e9,
+             "hbm_peak_gbs": peaks["hbm"]}
+
+    cpu = None
+    if not args.no_cpu_baseline and not big:
+        from oracle import hifa4_oracle as orc
+        orc.build()
+        qn, kn, vn = (t.float().numpy() for t in (qh, kh, vh))
+        sn = None if s is None else s.cpu().numpy()
+        isn = None if inv_s is None else inv_s.cpu().numpy()
+        t1, cores = oracle_time(cfg, qn, kn, vn, sn, isn, [0])
+        n_heads = max(1, min(cfg.Hq - 1, int(12.0 / max(t1, 1e-3))))
+        heads = [1 + int(i * (cfg.Hq - 1) / n_heads) for i in range(n_heads)]
+        t, cores = oracle_time(cfg, qn, kn, vn, sn, isn, heads)
+        cpu = {"value": n_heads * head_flops(cfg) / t / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"{n_heads} of {cfg.B * cfg.Hq} (batch, head) slices of {cfg.name}, all {cfg.N} rows each, "
+                         f"{t:.1f} s"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "N": cfg.N, "d": cfg.d,
+                       "causal": cfg.causal, "Br": 128, "Bc": cfg.Bc, "in_dtype": cfg.dtype, "out_dtype": "f32",
+                       "smooth_mode": cfg.smooth_mode, "step": "hifa4_quantize_qkv + hifa4_attention_fwd",
+                       "l2": "flushed between steps (256 MiB write), outside the per-step events",
+                       "parallelism": f"replicated batches x{world}"},
+            "frac_of_nominal_peak": {k_: value / world / v_ for k_, v_ in NOMINAL.items()},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
+            "quantize": quant, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
