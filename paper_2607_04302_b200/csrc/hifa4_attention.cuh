@@ -23,6 +23,8 @@ struct DebugReq {
 struct AttnArgs {
     int B, Hq, Hkv, N;
     int causal, out_dtype;
+    int dev_flags;                // development experiments only (0 in normal use)
+    long long* trace;             // development timeline buffer or nullptr
     float c0, c1;                 // sigma, sigma * log2(e)
     void* out;
     int* d_status;
@@ -53,68 +55,177 @@ struct Cfg {
 
 __device__ __forceinline__ float f16_round(float x) { return __half2float(__float2half_rn(x)); }
 
-// Quantize 64 softmax weights (already rounded to FP16, held as floats, all >= 0) to HIF4 and
-// write the BF16 image of P-hat into shared memory as row `row` of a 128-byte-swizzled tile.
-// Optionally dumps nibbles and subgroup steps.
-__device__ __forceinline__ void quantize_p64(const float (&p)[64], uint32_t p_sub_base, int row,
-                                             uint8_t* dump_codes, float* dump_step)
+// exp2 of two values, each result rounded to FP16 (one packed conversion) and widened back.
+__device__ __forceinline__ void exp2_f16_pair(float t0, float t1, float& e0, float& e1)
 {
-    float At[16];
-    float A = 0.f;
-#pragma unroll
-    for (int t = 0; t < 16; ++t) {
-        At[t] = fmaxf(fmaxf(p[4 * t], p[4 * t + 1]), fmaxf(p[4 * t + 2], p[4 * t + 3]));
-        A = fmaxf(A, At[t]);
-    }
-    const uint32_t row_base = p_sub_base + (row >> 3) * 1024 + (row & 7) * 128;
-    const int sw = row & 7;
+    const float a = ex2_approx(t0), b = ex2_approx(t1);
+    uint32_t h2;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(h2) : "f"(b), "f"(a));     // a -> low half, b -> high half
+    asm("{\n\t.reg .b16 lo, hi;\n\t"
+        "mov.b32 {lo, hi}, %2;\n\t"
+        "cvt.f32.f16 %0, lo;\n\t"
+        "cvt.f32.f16 %1, hi;\n\t}"
+        : "=f"(e0), "=f"(e1) : "r"(h2));
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// Quantize NU*8 consecutive softmax weights of one 64-key HIF4 group (already rounded to FP16,
+// held as floats, all >= 0) and return the BF16 image of P-hat as NU*4 packed words (element 2i
+// in the low half of word i).  A is the maximum of the whole group (the caller combines partial
+// maxima when a group is split over threads) and At[t] the maxima of this thread's 4-key
+// subgroups.  Optionally dumps nibbles and subgroup steps.
+//
+// Arithmetic (all exact): the element code is m = RNE(p / step).  q = RZ(p * (1/step)) lands
+// exactly on j + 1/2 for every tie (see e6m2_inv4), y = q + 1.5 * 2^23 rounds q to the nearest
+// integer with ties to even, and fma(y, step, -1.5 * 2^23 * step) = m * step without rounding.
+// The shift of a 4-key subgroup with maximum At is read off the float bit patterns:
+// n - 1 = max((bits(At) - bits(1.75 S) - 1) >> 23, -1); the pair rule "level-2 bit = 1 iff
+// max(need) = 2 or min(need) >= 1" is a = (n0 + n1 + 2) >> 2 and the shifts are max(n, a).
+template <int NU>
+__device__ __forceinline__ void quantize_p_units(const float (&p)[NU * 8], const float (&At)[NU * 2], float A,
+                                                 uint32_t (&w)[NU * 4], uint8_t* dump_codes, float* dump_step)
+{
     if (A == 0.f) {
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch)
-            asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(row_base + ((ch ^ sw) << 4)), "r"(0) : "memory");
+        for (int i = 0; i < NU * 4; ++i) w[i] = 0u;
         if (dump_codes) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) reinterpret_cast<uint4*>(dump_codes)[i] = make_uint4(0, 0, 0, 0);
+            for (int i = 0; i < NU / 2; ++i) reinterpret_cast<uint4*>(dump_codes)[i] = make_uint4(0, 0, 0, 0);
         }
         if (dump_step) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) reinterpret_cast<float4*>(dump_step)[i] = make_float4(0, 0, 0, 0);
+            for (int i = 0; i < NU / 2; ++i) reinterpret_cast<float4*>(dump_step)[i] = make_float4(0, 0, 0, 0);
         }
         return;
     }
     const int code = e6m2_code_for_max(A);
     const float S = e6m2_value(code);
-    const float inv4 = e6m2_inv4(code);
+    const uint32_t inv4_bits = __float_as_uint(e6m2_inv4(code));
+    const uint32_t s4_bits = __float_as_uint(S) - (2u << 23);              // S / 4
+    const int t1 = (int)__float_as_uint(1.75f * S) + 1;
+    const float MAGIC = 12582912.f;                                        // 1.5 * 2^23
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {                    // one level-2 unit = 8 keys = one 16-byte chunk
-        int a, b0, b1;
-        hif4_pair_bits(hif4_need(At[2 * u], S), hif4_need(At[2 * u + 1], S), a, b0, b1);
-        uint32_t w[4];
+    for (int u = 0; u < NU; ++u) {                   // one level-2 unit = 8 keys
+        const int n0 = max(((int)__float_as_uint(At[2 * u]) - t1) >> 23, -1);       // need - 1
+        const int n1 = max(((int)__float_as_uint(At[2 * u + 1]) - t1) >> 23, -1);
+        const int a = (n0 + n1 + 4) >> 2;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const int k = a + (h ? b1 : b0);
-            const float inv_step = scale_pow2(inv4, -k);
-            const float step = scale_pow2(S, k - 2);
+            const int k = max((h ? n1 : n0) + 1, a);
+            const float inv_step = __uint_as_float(inv4_bits - ((uint32_t)k << 23));
+            const float step = __uint_as_float(s4_bits + ((uint32_t)k << 23));
+            const float negc = -MAGIC * step;
             float v[4];
             uint32_t packed = 0;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int m = __float2int_rn(__fmul_rz(p[8 * u + 4 * h + i], inv_step));
-                v[i] = (float)m * step;
-                packed |= (uint32_t)m << (8 * i);
+                const float y = __fadd_rn(__fmul_rz(p[8 * u + 4 * h + i], inv_step), MAGIC);
+                v[i] = fmaf(y, step, negc);
+                if (dump_codes) packed |= (__float_as_uint(y) & 15u) << (8 * i);
             }
-            __nv_bfloat162 lo = __floats2bfloat162_rn(v[0], v[1]);
-            __nv_bfloat162 hi = __floats2bfloat162_rn(v[2], v[3]);
-            w[2 * h] = *reinterpret_cast<uint32_t*>(&lo);
-            w[2 * h + 1] = *reinterpret_cast<uint32_t*>(&hi);
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h]) : "f"(v[1]), "f"(v[0]));
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h + 1]) : "f"(v[3]), "f"(v[2]));
             if (dump_step) dump_step[2 * u + h] = step;
             if (dump_codes) reinterpret_cast<uint32_t*>(dump_codes)[2 * u + h] = packed;
         }
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                     ::"r"(row_base + ((u ^ sw) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
     }
 }
 
+// Fused form of Algorithm 1 lines 9-10 for NU*8 consecutive keys of one 64-key group: takes the raw
+// score accumulators (masked ones already -inf), forms P = exp2(acc * c1 - mL) rounded to FP16 and
+// quantizes it unit by unit, so that the exponentials (MUFU pipe) and the quantizer arithmetic
+// (ALU/FMA pipes) of a warp interleave.  A is the group maximum of P, which the caller gets from
+// the group maximum of the accumulators through the same instruction sequence
+// (p_of_score): that is exact because fma, ex2.approx (checked exhaustively over [-40, 0]) and
+// the FP16 rounding are all monotone non-decreasing.
+__device__ __forceinline__ float p_of_score(float acc, float c1, float mL)
+{
+    return f16_round(ex2_approx(fmaf(acc, c1, -mL)));
+}
+
+template <int NU>
+__device__ __forceinline__ void exp_quantize_units(const float (&acc)[NU * 8], float c1, float mL, float A,
+                                                   uint32_t (&w)[NU * 4], uint8_t* dump_codes, float* dump_step)
+{
+    if (A == 0.f) {
+#pragma unroll
+        for (int i = 0; i < NU * 4; ++i) w[i] = 0u;
+        if (dump_codes) {
+#pragma unroll
+            for (int i = 0; i < NU / 2; ++i) reinterpret_cast<uint4*>(dump_codes)[i] = make_uint4(0, 0, 0, 0);
+        }
+        if (dump_step) {
+#pragma unroll
+            for (int i = 0; i < NU / 2; ++i) reinterpret_cast<float4*>(dump_step)[i] = make_float4(0, 0, 0, 0);
+        }
+        return;
+    }
+    const int code = e6m2_code_for_max(A);
+    const float S = e6m2_value(code);
+    const uint32_t inv4_bits = __float_as_uint(e6m2_inv4(code));
+    const uint32_t s4_bits = __float_as_uint(S) - (2u << 23);              // S / 4
+    const int t1 = (int)__float_as_uint(1.75f * S) + 1;
+    const float MAGIC = 12582912.f;                                        // 1.5 * 2^23
+#pragma unroll
+    for (int u = 0; u < NU; ++u) {
+        float p[8];
+#pragma unroll
+        for (int i = 0; i < 8; i += 2)
+            exp2_f16_pair(fmaf(acc[8 * u + i], c1, -mL), fmaf(acc[8 * u + i + 1], c1, -mL), p[i], p[i + 1]);
+        const float At0 = fmaxf(max3(p[0], p[1], p[2]), p[3]);
+        const float At1 = fmaxf(max3(p[4], p[5], p[6]), p[7]);
+        const int n0 = max(((int)__float_as_uint(At0) - t1) >> 23, -1);       // need - 1
+        const int n1 = max(((int)__float_as_uint(At1) - t1) >> 23, -1);
+        const int a = (n0 + n1 + 4) >> 2;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int k = max((h ? n1 : n0) + 1, a);
+            const float inv_step = __uint_as_float(inv4_bits - ((uint32_t)k << 23));
+            const float step = __uint_as_float(s4_bits + ((uint32_t)k << 23));
+            const float negc = -MAGIC * step;
+            float v[4];
+            uint32_t packed = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float y = __fadd_rn(__fmul_rz(p[4 * h + i], inv_step), MAGIC);
+                v[i] = fmaf(y, step, negc);
+                if (dump_codes) packed |= (__float_as_uint(y) & 15u) << (8 * i);
+            }
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h]) : "f"(v[1]), "f"(v[0]));
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h + 1]) : "f"(v[3]), "f"(v[2]));
+            if (dump_step) dump_step[2 * u + h] = step;
+            if (dump_codes) reinterpret_cast<uint32_t*>(dump_codes)[2 * u + h] = packed;
+        }
+    }
+}
+
+// Whole 64-key group held by one thread; the image goes to row `row` of a 128-byte-swizzled
+// shared-memory tile (the layout a K-major tcgen05 operand descriptor with SWIZZLE_128B reads).
+__device__ __forceinline__ void quantize_p64(const float (&p)[64], uint32_t p_sub_base, int row,
+                                             uint8_t* dump_codes, float* dump_step)
+{
+    float At[16];
+#pragma unroll
+    for (int t = 0; t < 16; ++t) At[t] = fmaxf(max3(p[4 * t], p[4 * t + 1], p[4 * t + 2]), p[4 * t + 3]);
+    float A4[4];
+#pragma unroll
+    for (int t = 0; t < 4; ++t) A4[t] = fmaxf(max3(At[4 * t], At[4 * t + 1], At[4 * t + 2]), At[4 * t + 3]);
+    const float A = fmaxf(max3(A4[0], A4[1], A4[2]), A4[3]);
+    uint32_t w[32];
+    quantize_p_units<8>(p, At, A, w, dump_codes, dump_step);
+    const uint32_t row_base = p_sub_base + (row >> 3) * 1024 + (row & 7) * 128;
+    const int sw = row & 7;
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                     ::"r"(row_base + ((u ^ sw) << 4)), "r"(w[4 * u]), "r"(w[4 * u + 1]), "r"(w[4 * u + 2]), "r"(w[4 * u + 3]) : "memory");
+}
 
 // BF16 tensor [heads][rows][cols] (cols contiguous), box [1][box_rows][64 cols], 128-byte swizzle,
 // out-of-range elements read as zero.  Returns false if the driver entry point is unavailable or

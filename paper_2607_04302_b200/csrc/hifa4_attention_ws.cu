@@ -1,15 +1,23 @@
 // Warp-specialised HiFA4 attention forward for d = 128, Bc = 128 (Algorithm 1 lines 4-13).
 //
-// One CTA = 128 query rows of one (batch, query head), 10 warps:
-//   warps 0-7  softmax / quantize: warp w owns rows 32*(w%4).. of the tile and the 64-key HIF4
-//              group (w/4) of every 128-key tile, so a thread holds exactly one group of one row;
-//              the two threads of a row exchange their partial row maxima through shared memory
-//   warp 8     TMA producer: Q once, then K and V^T tiles through two-stage rings
-//   warp 9     tcgen05 issuer: S = Q K^T for tile j+1 is issued as soon as the softmax warps
-//              have pulled S(j) into registers, then [O | l] += P-hat(j) [V-hat | 1]
-// S lives in 128 tensor-memory columns, [O | l] in 144; P-hat goes through one swizzled
-// shared-memory tile.  Every wait is bounded; a wait that expires raises the abort flag, writes
-// the status word and every role falls through to the common exit (tensor memory is freed).
+// One CTA = 128 query rows of one (batch, query head), 4*KS + 2 warps (KS = 2 or 4):
+//   warps 0..4*KS-1  softmax / quantize: warp w owns rows 32*(w%4).. of the tile and keys
+//              (128/KS)*(w/4).. of every 128-key tile.  With KS = 2 a thread holds one whole
+//              64-key HIF4 group of one row; with KS = 4 half a group (4 level-2 units).  The
+//              threads of a row exchange their partial row maxima (and, for KS = 4, the two
+//              halves of a group their partial group maxima) through shared memory
+//   next warp  TMA producer: Q once, then K and V^T tiles through two-stage rings
+//   last warp  tcgen05 issuer
+// Tensor memory: [O | l] in columns 0..143, two S buffers of 128 columns.  S = Q K^T of tile j+2
+// is issued right after PV of tile j, so the tensor pipe always has work queued.  The softmax
+// warps pull S(j) into registers and write the BF16 image of P-hat(j) back over the first 64
+// columns of the same buffer; [O | l] += P-hat(j) [V-hat | 1] then takes its A operand from tensor
+// memory and V^T (with its rows of ones) from shared memory.  MMAs of one thread complete in issue
+// order, which is what makes the buffer reuse safe: S(j+2) is issued after PV(j).
+// Every wait is bounded; a wait that expires raises the abort flag, writes the status word and
+// every role falls through to the common exit (tensor memory is freed).
+#include <cstdio>
+#include <cstdlib>
 #include "hifa4_attention.cuh"
 
 namespace hifa4 {
@@ -20,41 +28,63 @@ constexpr int Q_BYTES = 2 * 16384;
 constexpr int K_STAGE = 2 * 16384;
 constexpr int V_CHUNK = (D + 16) * 128;
 constexpr int V_STAGE = 2 * V_CHUNK;
-constexpr int P_BYTES = 2 * 16384;
 constexpr int Q_OFF = 0;
 constexpr int K_OFF = Q_OFF + Q_BYTES;
 constexpr int V_OFF = K_OFF + STAGES * K_STAGE;
-constexpr int P_OFF = V_OFF + STAGES * V_STAGE;
-constexpr int MISC_OFF = P_OFF + P_BYTES;           // barriers, tmem slot, abort flag
-constexpr int XCHG_OFF = MISC_OFF + 256;            // [2 parities][2 groups][128 rows] floats
-constexpr int SMEM_BYTES = XCHG_OFF + 2 * 2 * 128 * 4 + 1024;
-constexpr int O_COLS = D + 16, S_COL = 256, TMEM_COLS = 512;
-constexpr int THREADS = 320;
-enum { BAR_Q = 0, BAR_KF = 1, BAR_KE = 3, BAR_VF = 5, BAR_VE = 7, BAR_SF = 9, BAR_SFREE = 10,
-       BAR_PF = 11, BAR_PV = 12, BAR_X = 13, N_BARS = 17 };
+constexpr int MISC_OFF = V_OFF + STAGES * V_STAGE;  // barriers, tmem slot, abort flag
+constexpr int XCHG_OFF = MISC_OFF + 256;            // row maxima [2 parities][4 splits][128 rows] floats,
+constexpr int XCHG_BYTES = 2 * 2 * 4 * 128 * 4;     // then group maxima, same shape
+constexpr int SMEM_BYTES = XCHG_OFF + XCHG_BYTES + 1024;
+constexpr int O_COLS = D + 16, QT_COL = 144, S_COL = 256, TMEM_COLS = 512;   // [O | l], Q image, 2 x S
+enum { BAR_Q = 0, BAR_KF = 1, BAR_KE = 3, BAR_VF = 5, BAR_VE = 7, BAR_SF = 9, BAR_PF = 11,
+       BAR_PV = 13, BAR_X = 14, BAR_XP = 18, BAR_QT = 26, N_BARS = 27 };
 }  // namespace ws
 
+__device__ int g_wait_mode;
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
-    for (uint32_t i = 0; i < (1u << 18); ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 255u && *abort_flag) return false;
+    if (g_wait_mode == 1) {
+        for (uint32_t i = 0; i < (1u << 22); ++i) {
+            if (mbar_try_wait(bar, parity)) return true;
+            if ((i & 1023u) == 1023u && *abort_flag) return false;
+        }
+        return false;
+    }
+    if (g_wait_mode == 2) {
+        for (uint32_t i = 0; i < (1u << 20); ++i) {
+            if (mbar_try_wait_hint(bar, parity, 500u)) return true;
+            if (*abort_flag) return false;
+        }
+        return false;
+    }
+    // at most 2^16 polls of up to 16 us each: about a second before giving up
+    for (uint32_t i = 0; i < (1u << 16); ++i) {
+        if (mbar_try_wait_hint(bar, parity, 16000u)) return true;
+        if (*abort_flag) return false;
     }
     return false;
 }
 
-__global__ void __launch_bounds__(ws::THREADS, 1)
+#define TRACE(slot) do { if (tr && jt < 24) tr[(jt) * 16 + (slot)] = clock64(); } while (0)
+
+template <int KS>
+__global__ void __launch_bounds__((4 * KS + 2) * 32, 1)
 attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                         const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnArgs args)
 {
     using namespace ws;
+    constexpr int NSW = 4 * KS;                 // softmax warps
+    constexpr int THREADS = (NSW + 2) * 32;
+    constexpr int W_TMA = NSW, W_MMA = NSW + 1;
+    constexpr int KPT = BC / KS;                // keys per thread and tile
+    constexpr int NU = KPT / 8;                 // level-2 units per thread
     if (args.d_status && *reinterpret_cast<volatile int*>(args.d_status) != 0) return;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     const uint32_t q_s = smem_base + Q_OFF, k_s = smem_base + K_OFF, v_s = smem_base + V_OFF,
-                   p_s = smem_base + P_OFF, bars = smem_base + MISC_OFF;
+                   bars = smem_base + MISC_OFF;
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + MISC_OFF + 8 * N_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + MISC_OFF + 8 * N_BARS + 8);
@@ -78,13 +108,14 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             mbar_init(bar(BAR_KF + s), 1); mbar_init(bar(BAR_KE + s), 1);
             mbar_init(bar(BAR_VF + s), 1); mbar_init(bar(BAR_VE + s), 1);
         }
-        mbar_init(bar(BAR_SF), 1); mbar_init(bar(BAR_SFREE), 8);
-        mbar_init(bar(BAR_PF), 8); mbar_init(bar(BAR_PV), 1);
-        for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_X + i), 2);
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(BAR_SF + i), 1); mbar_init(bar(BAR_PF + i), NSW); }
+        mbar_init(bar(BAR_PV), 1); mbar_init(bar(BAR_QT), NSW);
+        for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_X + i), KS);
+        for (int i = 0; i < 8; ++i) mbar_init(bar(BAR_XP + i), 2);
         fence_barrier_init();
     }
-    if (warp == 9) { tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS); tmem_relinquish(); }
-    if (warp == 8 && lane == 0) { tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_k); tma_prefetch_desc(&tmap_v); }
+    if (warp == W_MMA) { tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS); tmem_relinquish(); }
+    if (warp == W_TMA && lane == 0) { tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_k); tma_prefetch_desc(&tmap_v); }
     for (int i = tid; i < STAGES * 2 * 128; i += THREADS) {      // ones rows under every V^T chunk
         const int chunk = i / 128, off = (i % 128) * 16;
         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};"
@@ -101,7 +132,7 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         if (args.d_status) atomicCAS(args.d_status, 0, HIFA4_ERR_TIMEOUT + 16 * site);
     };
 
-    if (warp == 8) {
+    if (warp == W_TMA) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             mbar_expect_tx(bar(BAR_Q), Q_BYTES);
@@ -112,68 +143,106 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
                 const int j0 = jt * BC;
                 if (!wait_or_abort(bar(BAR_KE + st), ph ^ 1u, abort_flag)) { fail(1); break; }
+                if ((args.dev_flags & 64) && jt >= 2) { mbar_arrive(bar(BAR_KF + st)); } else {
                 mbar_expect_tx(bar(BAR_KF + st), K_STAGE);
                 tma_load_3d(k_s + st * K_STAGE, &tmap_k, bar(BAR_KF + st), 0, j0, bh_kv);
-                tma_load_3d(k_s + st * K_STAGE + 16384, &tmap_k, bar(BAR_KF + st), 64, j0, bh_kv);
+                tma_load_3d(k_s + st * K_STAGE + 16384, &tmap_k, bar(BAR_KF + st), 64, j0, bh_kv); }
                 if (!wait_or_abort(bar(BAR_VE + st), ph ^ 1u, abort_flag)) { fail(2); break; }
+                if ((args.dev_flags & 64) && jt >= 2) { mbar_arrive(bar(BAR_VF + st)); } else {
                 mbar_expect_tx(bar(BAR_VF + st), 2 * D * 128);
                 tma_load_3d(v_s + st * V_STAGE, &tmap_v, bar(BAR_VF + st), j0, 0, bh_kv);
-                tma_load_3d(v_s + st * V_STAGE + V_CHUNK, &tmap_v, bar(BAR_VF + st), j0 + 64, 0, bh_kv);
+                tma_load_3d(v_s + st * V_STAGE + V_CHUNK, &tmap_v, bar(BAR_VF + st), j0 + 64, 0, bh_kv); }
             }
         }
-    } else if (warp == 9) {
+    } else if (warp == W_MMA) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc_s = umma_idesc_bf16(128, BC);
             constexpr uint32_t idesc_o = umma_idesc_bf16(128, O_COLS);
-            auto issue_qk = [&](int jt) {
+            const uint32_t k_lo = umma_desc_lo(k_s), v_lo = umma_desc_lo(v_s);
+            long long* tr = (args.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) ? args.trace : nullptr;
+            auto issue_qk = [&](int jt) {                 // S(jt) -> buffer jt % 2, K stage jt % 2
                 const int st = jt & 1;
+                const uint32_t d = tmem + S_COL + st * 128;
+                const uint32_t b0 = k_lo + st * (K_STAGE >> 4);
 #pragma unroll
-                for (int s = 0; s < 2; ++s)
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        umma_bf16_ss(tmem + S_COL, umma_desc_sw128(q_s + s * 16384 + kk * 32),
-                                     umma_desc_sw128(k_s + st * K_STAGE + s * 16384 + kk * 32), idesc_s,
-                                     (s | kk) ? 1u : 0u);
-                umma_commit(bar(BAR_SF));
+                for (int kk = 0; kk < 8; ++kk)               // A = Q image in tensor memory, 8 columns per 16 channels
+                    umma_bf16_ts_lo(d, tmem + QT_COL + kk * 8, b0 + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2, idesc_s,
+                                    kk ? 1u : 0u);
+                umma_commit(bar(BAR_SF + st));
                 umma_commit(bar(BAR_KE + st));
             };
-            bool ok = wait_or_abort(bar(BAR_Q), 0, abort_flag) && wait_or_abort(bar(BAR_KF), 0, abort_flag);
+            bool ok = wait_or_abort(bar(BAR_QT), 0, abort_flag);
+            for (int jt = 0; ok && jt < min(2, n_tiles); ++jt) {
+                ok = wait_or_abort(bar(BAR_KF + jt), 0, abort_flag);
+                if (ok) { tc_fence_after(); issue_qk(jt); }
+            }
             if (!ok) fail(3);
             if (ok) {
-                tc_fence_after();
-                issue_qk(0);
                 for (int jt = 0; jt < n_tiles; ++jt) {
-                    if (jt + 1 < n_tiles) {
-                        const int st1 = (jt + 1) & 1;
-                        if (!wait_or_abort(bar(BAR_KF + st1), (uint32_t)((jt + 1) >> 1) & 1u, abort_flag)) { fail(4); break; }
-                        if (!wait_or_abort(bar(BAR_SFREE), (uint32_t)jt & 1u, abort_flag)) { fail(5); break; }
-                        tc_fence_after();
-                        issue_qk(jt + 1);
-                    }
                     const int st = jt & 1;
-                    if (!wait_or_abort(bar(BAR_VF + st), (uint32_t)(jt >> 1) & 1u, abort_flag)) { fail(6); break; }
-                    if (!wait_or_abort(bar(BAR_PF), (uint32_t)jt & 1u, abort_flag)) { fail(7); break; }
+                    const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
+                    if (!wait_or_abort(bar(BAR_VF + st), ph, abort_flag)) { fail(6); break; }
+                    if (!(args.dev_flags & 128)) if (!wait_or_abort(bar(BAR_PF + st), ph, abort_flag)) { fail(7); break; }
                     tc_fence_after();
+                    TRACE(0);
+                    // PV(jt) and QK(jt+2) accumulate into different tensor-memory regions; their k-steps are
+                    // issued interleaved so that consecutive MMAs never depend on each other
+                    const bool more = jt + 2 < n_tiles;
+                    if (more) {
+                        if (!wait_or_abort(bar(BAR_KF + st), (uint32_t)((jt + 2) >> 1) & 1u, abort_flag)) { fail(4); break; }
+                        tc_fence_after();
+                    }
+                    {
+                        const uint32_t a0 = tmem + S_COL + st * 128;
+                        const uint32_t b0 = v_lo + st * (V_STAGE >> 4);
+                        const uint32_t kb0 = k_lo + st * (K_STAGE >> 4);
+                        // P-hat(jt) sits in columns 0..63 of S buffer st: S(jt+2) may only overwrite columns
+                        // whose P-hat k-step has already been issued, so QK trails PV by the whole tile
+                        if (args.dev_flags & 256) {
 #pragma unroll
-                    for (int c = 0; c < 2; ++c)
+                            for (int kk = 0; kk < 8; ++kk) {
+                                umma_bf16_ts_lo(tmem, a0 + kk * 8, b0 + (kk >> 2) * (V_CHUNK >> 4) + (kk & 3) * 2, idesc_o,
+                                                (jt > 0 || kk > 0) ? 1u : 0u);
+                                if (more)
+                                    umma_bf16_ts_lo(a0, tmem + QT_COL + kk * 8, kb0 + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2,
+                                                    idesc_s, kk ? 1u : 0u);
+                            }
+                        } else {
+                            if (!(args.dev_flags & 512))
 #pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            umma_bf16_ss(tmem, umma_desc_sw128(p_s + c * 16384 + kk * 32),
-                                         umma_desc_sw128(v_s + st * V_STAGE + c * V_CHUNK + kk * 32), idesc_o,
-                                         (jt > 0 || c > 0 || kk > 0) ? 1u : 0u);
+                            for (int kk = 0; kk < 8; ++kk)
+                                umma_bf16_ts_lo(tmem, a0 + kk * 8, b0 + (kk >> 2) * (V_CHUNK >> 4) + (kk & 3) * 2, idesc_o,
+                                                (jt > 0 || kk > 0) ? 1u : 0u);
+                            if (more && !(args.dev_flags & 1024)) {
+#pragma unroll
+                                for (int kk = 0; kk < 8; ++kk)
+                                    umma_bf16_ts_lo(a0, tmem + QT_COL + kk * 8, kb0 + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2,
+                                                    idesc_s, kk ? 1u : 0u);
+                            }
+                        }
+                    }
+                    TRACE(1);
                     umma_commit(bar(BAR_PV));
                     umma_commit(bar(BAR_VE + st));
+                    if (more) {
+                        umma_commit(bar(BAR_SF + st));
+                        umma_commit(bar(BAR_KE + st));
+                    }
                 }
             }
         }
     } else {
         // ------------------------------------------------------------------ softmax / quantize
-        const int wg = warp >> 2, quarter = warp & 3;
-        const int r_loc = quarter * 32 + lane;                     // row inside the tile = TMEM lane
+        const int kq = warp >> 2, quarter = warp & 3;             // key split, row quarter
+        const int gq = (kq * KPT) / 64;                           // 64-key group inside the tile
+        const int r_loc = quarter * 32 + lane;                    // row inside the tile = TMEM lane
         const int row = q0 + r_loc;
         const uint32_t t_lane = tmem + ((uint32_t)(quarter * 32) << 16);
         const uint32_t xbar = bar(BAR_X + quarter);
+        const uint32_t xpbar = bar(BAR_XP + quarter * 2 + gq);
+        float* xmax = xchg;                                       // [2][4][128] partial row maxima of S
+        float* xpm = xchg + 2 * 4 * 128;                          // [2][4][128] partial group maxima of P
         const float LOG2E = 1.4426950408889634f;
         const int key_lim = args.causal ? min(row, N - 1) : N - 1;
         int dbg_slot = -1;
@@ -182,61 +251,94 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 dbg_slot = i;
         float m_run = -INFINITY;
         bool ok = true;
+        long long* tr = (args.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && warp == 0 && lane == 0) ? args.trace : nullptr;
 
-        for (int jt = 0; jt < n_tiles; ++jt) {
-            const int j0 = jt * BC;
-            const uint32_t par = (uint32_t)jt & 1u;
-            if (!wait_or_abort(bar(BAR_SF), par, abort_flag)) { fail(8); ok = false; break; }
-            tc_fence_after();
-            float p[64];
-            {
-                uint32_t r0[32], r1[32];
-                tmem_ld32(t_lane + S_COL + wg * 64, r0);
-                tmem_ld32(t_lane + S_COL + wg * 64 + 32, r1);
-                tmem_wait_ld();
+        // Q-hat image: shared memory (swizzled TMA tile) -> tensor memory, so that S = Q K^T reads its A
+        // operand from tensor memory and only K from shared memory.  This thread moves channels
+        // 128/NSW*... of its row: 128 / KS channels = 64 / KS columns of packed BF16 pairs.
+        if (wait_or_abort(bar(BAR_Q), 0, abort_flag)) {
+            constexpr int QC = 64 / KS;                            // columns per thread
+            uint32_t qw[QC];
+            const int sw = r_loc & 7;
 #pragma unroll
-                for (int i = 0; i < 32; ++i) { p[i] = __uint_as_float(r0[i]); p[32 + i] = __uint_as_float(r1[i]); }
+            for (int c = 0; c < QC / 4; ++c) {
+                const int chunk = kq * (QC / 4) + c;               // 16-byte chunk of the 256-byte row
+                const uint32_t a = q_s + (chunk >> 3) * 16384 + (r_loc >> 3) * 1024 + sw * 128 + (((chunk & 7) ^ sw) << 4);
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(qw[4 * c]), "=r"(qw[4 * c + 1]), "=r"(qw[4 * c + 2]), "=r"(qw[4 * c + 3]) : "r"(a));
             }
+            if constexpr (KS == 2) tmem_st32(t_lane + QT_COL + kq * QC, qw);
+            else tmem_st16(t_lane + QT_COL + kq * QC, qw);
+            tmem_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_SFREE));
+            if (lane == 0) mbar_arrive(bar(BAR_QT));
+        } else { fail(13); ok = false; }
 
-            // row maximum over the 128-key tile (line 7): own 64 keys, then the partner's
-            const bool need_mask = (args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N);
-            const int kbase = j0 + wg * 64;
-            float mx = -INFINITY;
-            if (need_mask) {
+        for (int jt = 0; ok && jt < n_tiles; ++jt) {
+            const int j0 = jt * BC;
+            const uint32_t par = (uint32_t)jt & 1u;
+            const int sb = jt & 1;                             // S / P-hat buffer and its barrier pair
+            const uint32_t ph2 = (uint32_t)(jt >> 1) & 1u;
+            const uint32_t t_s = t_lane + S_COL + sb * 128;
+            if (!wait_or_abort(bar(BAR_SF + sb), ph2, abort_flag)) { fail(8); ok = false; break; }
+            tc_fence_after();
+            TRACE(2);
+            float p[KPT];
 #pragma unroll
-                for (int i = 0; i < 64; ++i) mx = fmaxf(mx, (kbase + i > key_lim) ? -INFINITY : p[i]);
-            } else {
+            for (int cc = 0; cc < KPT / 32; ++cc) {
+                uint32_t r[32];
+                tmem_ld32(t_s + kq * KPT + cc * 32, r);
+                tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 64; ++i) mx = fmaxf(mx, p[i]);
+                for (int i = 0; i < 32; ++i) p[cc * 32 + i] = __uint_as_float(r[i]);
             }
-            xchg[(par * 2 + wg) * 128 + r_loc] = mx;
+
+            TRACE(3);
+            // row maximum over the 128-key tile (line 7): own keys, then the other splits'
+            const bool need_mask = (args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N);
+            const int kbase = j0 + kq * KPT;
+            if (need_mask) {                                   // masked scores become -inf: exp gives exact zeros
+#pragma unroll
+                for (int i = 0; i < KPT; ++i) p[i] = (kbase + i > key_lim) ? -INFINITY : p[i];
+            }
+            float mx;
+            {
+                float t4[KPT / 4];
+#pragma unroll
+                for (int i = 0; i < KPT / 4; ++i) t4[i] = fmaxf(max3(p[4 * i], p[4 * i + 1], p[4 * i + 2]), p[4 * i + 3]);
+#pragma unroll
+                for (int w = KPT / 8; w >= 1; w >>= 1)
+#pragma unroll
+                    for (int i = 0; i < w; ++i) t4[i] = fmaxf(t4[i], t4[i + w]);
+                mx = t4[0];
+            }
+            const float mx_own = mx;
+            xmax[(par * 4 + kq) * 128 + r_loc] = mx;
+            tc_fence_before();                                 // S(jt) is in registers: others may overwrite it with P-hat
             __syncwarp();
             if (lane == 0) mbar_arrive(xbar);
-            if (!wait_or_abort(xbar, par, abort_flag)) { fail(9); ok = false; break; }
-            mx = fmaxf(mx, xchg[(par * 2 + (wg ^ 1)) * 128 + r_loc]);
+            if (!(args.dev_flags & 8)) if (!wait_or_abort(xbar, par, abort_flag)) { fail(9); ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int o = 1; o < KS; ++o) mx = fmaxf(mx, xmax[(par * 4 + ((kq + o) % KS)) * 128 + r_loc]);
 
+            TRACE(4);
             const float m_new = fmaxf(m_run, f16_round(mx * args.c0));
             float rsc = 1.f;
             if (jt > 0 && m_new != m_run) rsc = f16_round(ex2_approx((m_run - m_new) * LOG2E));
             m_run = m_new;
             const float mL = m_run * LOG2E;
 
-            // P = exp(S - m) in FP16 (line 9)
-#pragma unroll
-            for (int i = 0; i < 64; ++i) {
-                float e = f16_round(ex2_approx(fmaf(p[i], args.c1, -mL)));
-                if (need_mask && (kbase + i > key_lim)) e = 0.f;
-                p[i] = e;
-            }
-            // the P tile and the O accumulator are free once PV(jt-1) has completed
-            if (jt > 0) {
-                if (!wait_or_abort(bar(BAR_PV), par ^ 1u, abort_flag)) { fail(10); ok = false; break; }
-                tc_fence_after();
-            }
-            // P-hat = HIF4(P) (line 10) -> BF16 image in the swizzled P tile
+            // group maximum of the scores: own keys and, when a 64-key group is split over two threads,
+            // the other half's partial maximum (already published for the row maximum)
+            float gmax = mx_own;
+            if (KS == 4) gmax = fmaxf(gmax, xmax[(par * 4 + (kq ^ 1)) * 128 + r_loc]);
+            const float A = p_of_score(gmax, args.c1, mL);         // = max of P over the group (monotone map)
+            TRACE(5);
+            TRACE(6);
+            // P = exp(S - m) in FP16 (line 9), P-hat = HIF4(P) (line 10); the BF16 image overwrites the
+            // first 64 columns of S(jt)
             uint8_t* dc = nullptr;
             float* ds = nullptr;
             if (dbg_slot >= 0 && row < N && kbase < N) {
@@ -244,13 +346,22 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 if (args.dbg.p_codes) dc = args.dbg.p_codes + r_idx * N + kbase;
                 if (args.dbg.p_step) ds = args.dbg.p_step + r_idx * (N / 4) + kbase / 4;
             }
-            quantize_p64(p, p_s + wg * 16384, r_loc, dc, ds);
-            fence_proxy_async_smem();
-            // rescale history (line 8); group 0 owns columns 0..79 of [O | l], group 1 columns 80..143
-            if (__any_sync(0xffffffffu, rsc != 1.f)) {
-                const uint32_t t_o = t_lane + (wg ? 80 : 0);
+            {
+                uint32_t w[NU * 4];
+                exp_quantize_units<NU>(p, args.c1, mL, A, w, dc, ds);
+                if constexpr (KS == 2) tmem_st32(t_s + kq * (KPT / 2), w);
+                else tmem_st16(t_s + kq * (KPT / 2), w);
+            }
+            TRACE(7);
+            // rescale history (line 8): the KS splits share the 144 columns of [O | l]
+            // (needs PV(jt-1) complete; a tile that leaves every maximum of the warp unchanged skips it)
+            if (!(args.dev_flags & 4) && __any_sync(0xffffffffu, rsc != 1.f)) {
+                if (!wait_or_abort(bar(BAR_PV), par ^ 1u, abort_flag)) { fail(10); ok = false; break; }
+                tc_fence_after();
+                constexpr int CW = O_COLS / KS;                // 72 or 36 columns per split
+                const uint32_t t_o = t_lane + kq * CW;
 #pragma unroll
-                for (int cc = 0; cc < 2; ++cc) {
+                for (int cc = 0; cc < CW / 32; ++cc) {
                     uint32_t r[32];
                     tmem_ld32(t_o + cc * 32, r);
                     tmem_wait_ld();
@@ -258,38 +369,50 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                     for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * rsc);
                     tmem_st32(t_o + cc * 32, r);
                 }
-                if (wg == 0) {
-                    uint32_t r[16];
-                    tmem_ld16(t_o + 64, r);
+                if (KS == 2) {
+                    uint32_t r[4];
+#pragma unroll
+                    for (int cc = 0; cc < 2; ++cc) {
+                        tmem_ld4(t_o + 64 + cc * 4, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * rsc);
+                        tmem_st4(t_o + 64 + cc * 4, r);
+                    }
+                } else {
+                    uint32_t r[4];
+                    tmem_ld4(t_o + 32, r);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * rsc);
-                    tmem_st16(t_o + 64, r);
+                    for (int i = 0; i < 4; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * rsc);
+                    tmem_st4(t_o + 32, r);
                 }
-                tmem_wait_st();
             }
+            TRACE(8);
+            tmem_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_PF));
+            if (lane == 0) mbar_arrive(bar(BAR_PF + sb));
+            TRACE(9);
         }
 
-        // finalize: out = O / l with l rounded to FP16 (line 13); group g writes channels 64g..64g+63
+        // finalize: out = O / l with l rounded to FP16 (line 13); split kq writes channels KPT*kq..
         if (ok && wait_or_abort(bar(BAR_PV), (uint32_t)(n_tiles - 1) & 1u, abort_flag)) {
             tc_fence_after();
-            uint32_t lr[16];
-            tmem_ld16(t_lane + D, lr);
+            uint32_t lr[4];
+            tmem_ld4(t_lane + D, lr);
             tmem_wait_ld();
             const float ell = __uint_as_float(lr[0]);
             const float l16 = f16_round(ell);
-            if (dbg_slot >= 0 && row < N && wg == 0) {
+            if (dbg_slot >= 0 && row < N && kq == 0) {
                 if (args.dbg.l_out) args.dbg.l_out[dbg_slot * 128 + r_loc] = ell;
                 if (args.dbg.m_out) args.dbg.m_out[dbg_slot * 128 + r_loc] = m_run;
             }
-            const size_t orow = ((size_t)bh_q * N + row) * D + wg * 64;
+            const size_t orow = ((size_t)bh_q * N + row) * D + kq * KPT;
 #pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
+            for (int cc = 0; cc < KPT / 32; ++cc) {
                 uint32_t r[32];
-                tmem_ld32(t_lane + wg * 64 + cc * 32, r);
+                tmem_ld32(t_lane + kq * KPT + cc * 32, r);
                 tmem_wait_ld();
                 if (row < N) {
                     float o[32];
@@ -324,7 +447,7 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
+    if (warp == W_MMA) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
 }
 
 int launch_attention_ws(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
@@ -333,15 +456,36 @@ int launch_attention_ws(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnA
     if (!make_bf16_map(&mq, qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, ws::D, 128)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, ws::D, ws::BC)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, ws::D, sh.N, ws::D)) return HIFA4_ERR_CUDA;
+    constexpr int KS = 4;
+    { const char* e = getenv("HIFA4_WAIT_MODE"); int m = e ? atoi(e) : 0; cudaMemcpyToSymbol(g_wait_mode, &m, sizeof(int)); }
+    auto kern = attention_fwd_ws_kernel<KS>;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(attention_fwd_ws_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 ws::SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ws::SMEM_BYTES) != cudaSuccess)
             return HIFA4_ERR_CUDA;
         attr_set = true;
     }
     dim3 grid((sh.N + 127) / 128, sh.Hq, sh.B);
-    attention_fwd_ws_kernel<<<grid, ws::THREADS, ws::SMEM_BYTES, st>>>(mq, mk, mv, args);
+    AttnArgs a2 = args;
+    static long long* d_trace = nullptr;
+    const bool want_trace = getenv("HIFA4_TRACE") != nullptr;
+    if (want_trace) {
+        if (!d_trace) cudaMalloc(&d_trace, 24 * 16 * 8);
+        cudaMemset(d_trace, 0, 24 * 16 * 8);
+        a2.trace = d_trace;
+    }
+    kern<<<grid, (4 * KS + 2) * 32, ws::SMEM_BYTES, st>>>(mq, mk, mv, a2);
+    if (want_trace) {
+        long long h[24 * 16];
+        cudaDeviceSynchronize();
+        cudaMemcpy(h, d_trace, sizeof(h), cudaMemcpyDeviceToHost);
+        long long t0 = h[2];
+        for (int j = 0; j < 24; ++j) {
+            fprintf(stderr, "tile %2d:", j);
+            for (int k = 0; k < 10; ++k) fprintf(stderr, " %7lld", h[j * 16 + k] ? h[j * 16 + k] - t0 : -1);
+            fprintf(stderr, "\n");
+        }
+    }
     count_launch();
     return cudaGetLastError() == cudaSuccess ? HIFA4_OK : HIFA4_ERR_CUDA;
 }
