@@ -7,7 +7,6 @@
 // 64 keys in registers and writes the BF16 image of P-hat into the swizzled shared-memory tile
 // the PV MMA consumes.  V^T tiles carry 16 extra rows of ones, so column d of the PV accumulator
 // is the row sum of P-hat: the normalizer of P-Reordering comes out of the same MMA.
-#include <cstdlib>
 #include "hifa4_attention.cuh"
 
 namespace hifa4 {
@@ -323,7 +322,6 @@ int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv&
     memset(&a, 0, sizeof(a));
     a.B = sh.B; a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.N = sh.N;
     a.causal = prm.causal ? 1 : 0;
-    { const char* e = getenv("HIFA4_DEV_FLAGS"); a.dev_flags = e ? atoi(e) : 0; }
     a.out_dtype = prm.out_dtype;
     const double sigma = prm.softmax_scale != 0.f ? (double)prm.softmax_scale : 1.0 / sqrt((double)sh.d);
     a.c0 = (float)sigma;

@@ -23,8 +23,6 @@ struct DebugReq {
 struct AttnArgs {
     int B, Hq, Hkv, N;
     int causal, out_dtype;
-    int dev_flags;                // development experiments only (0 in normal use)
-    long long* trace;             // development timeline buffer or nullptr
     float c0, c1;                 // sigma, sigma * log2(e)
     void* out;
     int* d_status;
@@ -149,58 +147,81 @@ __device__ __forceinline__ float p_of_score(float acc, float c1, float mL)
     return f16_round(ex2_approx(fmaf(acc, c1, -mL)));
 }
 
-template <int NU>
+// Arithmetic of the fused form (all exact except the exponential itself):
+//   q = RZ(p * (4/S))            group-constant multiplier; exactly j + 1/2 (in units of the finest
+//                                step S/4) on every rounding tie (see e6m2_inv4)
+//   y = q + 1.5 * 2^(23+k)       rounds q to the nearest multiple of 2^k, ties to the even multiple:
+//                                y - magic = m * 2^k with m the element code under shift k
+//   v = fma(y, S/4, -magic*S/4)  = m * 2^k * S/4, the dequantized value, no rounding
+// The shift k of a 4-key subgroup with maximum At is read off float bit patterns:
+//   need = max(bits(At) - bits(1.75 S) - 1 + 2^23, 0) >> 23   (0, 1 or 2)
+// and the pair rule "level-2 bit = 1 iff max(need) = 2 or min(need) >= 1" is a = (n0 + n1 + 2) >> 2,
+// k = max(need, a).  Multiplications, additions and FMAs run two elements at a time (f32x2).
+template <int NU, bool DBG>
 __device__ __forceinline__ void exp_quantize_units(const float (&acc)[NU * 8], float c1, float mL, float A,
                                                    uint32_t (&w)[NU * 4], uint8_t* dump_codes, float* dump_step)
 {
     if (A == 0.f) {
 #pragma unroll
         for (int i = 0; i < NU * 4; ++i) w[i] = 0u;
-        if (dump_codes) {
+        if (DBG) {
+            if (dump_codes) {
 #pragma unroll
-            for (int i = 0; i < NU / 2; ++i) reinterpret_cast<uint4*>(dump_codes)[i] = make_uint4(0, 0, 0, 0);
-        }
-        if (dump_step) {
+                for (int i = 0; i < NU / 2; ++i) reinterpret_cast<uint4*>(dump_codes)[i] = make_uint4(0, 0, 0, 0);
+            }
+            if (dump_step) {
 #pragma unroll
-            for (int i = 0; i < NU / 2; ++i) reinterpret_cast<float4*>(dump_step)[i] = make_float4(0, 0, 0, 0);
+                for (int i = 0; i < NU / 2; ++i) reinterpret_cast<float4*>(dump_step)[i] = make_float4(0, 0, 0, 0);
+            }
         }
         return;
     }
     const int code = e6m2_code_for_max(A);
     const float S = e6m2_value(code);
-    const uint32_t inv4_bits = __float_as_uint(e6m2_inv4(code));
-    const uint32_t s4_bits = __float_as_uint(S) - (2u << 23);              // S / 4
-    const int t1 = (int)__float_as_uint(1.75f * S) + 1;
-    const float MAGIC = 12582912.f;                                        // 1.5 * 2^23
+    const float inv4 = e6m2_inv4(code);
+    const float S4 = __uint_as_float(__float_as_uint(S) - (2u << 23));     // S / 4
+    const int tadd = (1 << 23) - ((int)__float_as_uint(1.75f * S) + 1);
+    const uint32_t MAGIC_BITS = 0x4B400000u;                               // 1.5 * 2^23
+    const uint32_t c0_bits = __float_as_uint(-12582912.f * S4);            // -magic * S/4 at shift 0
+    const uint64_t c1c1 = pack2(c1, c1), nml = pack2(-mL, -mL);
+    const uint64_t inv44 = pack2(inv4, inv4), s44 = pack2(S4, S4);
 #pragma unroll
     for (int u = 0; u < NU; ++u) {
         float p[8];
 #pragma unroll
-        for (int i = 0; i < 8; i += 2)
-            exp2_f16_pair(fmaf(acc[8 * u + i], c1, -mL), fmaf(acc[8 * u + i + 1], c1, -mL), p[i], p[i + 1]);
+        for (int i = 0; i < 8; i += 2) {
+            float t0, t1;
+            unpack2(fma2(pack2(acc[8 * u + i], acc[8 * u + i + 1]), c1c1, nml), t0, t1);
+            exp2_f16_pair(t0, t1, p[i], p[i + 1]);
+        }
         const float At0 = fmaxf(max3(p[0], p[1], p[2]), p[3]);
         const float At1 = fmaxf(max3(p[4], p[5], p[6]), p[7]);
-        const int n0 = max(((int)__float_as_uint(At0) - t1) >> 23, -1);       // need - 1
-        const int n1 = max(((int)__float_as_uint(At1) - t1) >> 23, -1);
-        const int a = (n0 + n1 + 4) >> 2;
+        const int n0 = max((int)__float_as_uint(At0) + tadd, 0) >> 23;
+        const int n1 = max((int)__float_as_uint(At1) + tadd, 0) >> 23;
+        const int a = (n0 + n1 + 2) >> 2;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            const int k = max((h ? n1 : n0) + 1, a);
-            const float inv_step = __uint_as_float(inv4_bits - ((uint32_t)k << 23));
-            const float step = __uint_as_float(s4_bits + ((uint32_t)k << 23));
-            const float negc = -MAGIC * step;
-            float v[4];
-            uint32_t packed = 0;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float y = __fadd_rn(__fmul_rz(p[4 * h + i], inv_step), MAGIC);
-                v[i] = fmaf(y, step, negc);
-                if (dump_codes) packed |= (__float_as_uint(y) & 15u) << (8 * i);
+            const uint32_t ks = (uint32_t)max(h ? n1 : n0, a) << 23;
+            const float magic = __uint_as_float(MAGIC_BITS + ks);
+            const float ck = __uint_as_float(c0_bits + ks);
+            const uint64_t mm = pack2(magic, magic), cc = pack2(ck, ck);
+            float v0, v1, v2, v3;
+            const uint64_t y01 = add2(mul2_rz(pack2(p[4 * h], p[4 * h + 1]), inv44), mm);
+            const uint64_t y23 = add2(mul2_rz(pack2(p[4 * h + 2], p[4 * h + 3]), inv44), mm);
+            unpack2(fma2(y01, s44, cc), v0, v1);
+            unpack2(fma2(y23, s44, cc), v2, v3);
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h]) : "f"(v1), "f"(v0));
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h + 1]) : "f"(v3), "f"(v2));
+            if (DBG) {
+                float y0, y1, y2, y3;
+                unpack2(y01, y0, y1);
+                unpack2(y23, y2, y3);
+                if (dump_step) dump_step[2 * u + h] = __uint_as_float(__float_as_uint(S4) + ks);
+                if (dump_codes)
+                    reinterpret_cast<uint32_t*>(dump_codes)[2 * u + h] =
+                        (__float_as_uint(y0) & 15u) | ((__float_as_uint(y1) & 15u) << 8) |
+                        ((__float_as_uint(y2) & 15u) << 16) | ((__float_as_uint(y3) & 15u) << 24);
             }
-            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h]) : "f"(v[1]), "f"(v[0]));
-            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h + 1]) : "f"(v[3]), "f"(v[2]));
-            if (dump_step) dump_step[2 * u + h] = step;
-            if (dump_codes) reinterpret_cast<uint32_t*>(dump_codes)[2 * u + h] = packed;
         }
     }
 }
