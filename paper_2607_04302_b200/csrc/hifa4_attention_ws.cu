@@ -40,11 +40,26 @@ enum { BAR_Q = 0, BAR_KF = 1, BAR_KE = 3, BAR_VF = 5, BAR_VE = 7, BAR_SF = 9, BA
 constexpr uint32_t WAIT_POLLS = 1u << 20;           // each poll blocks for a hardware-defined slice
 }  // namespace ws
 
+// Bounded waits.  wait_or_abort polls back to back (softmax warps: their waits are usually already
+// satisfied, and a late wake-up would sit on the critical path).  wait_sleepy lets the hardware
+// suspend the thread for up to a few microseconds per poll (it wakes when the phase completes), so
+// the producer and issuer warps, which wait most of the time, do not burn the issue slots and the
+// memory-I/O queue that the softmax warps need.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
-    for (uint32_t i = 0; i < ws::WAIT_POLLS; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 63u) == 63u && *abort_flag) return false;
+    for (uint32_t i = 0; i < ws::WAIT_POLLS / 64; ++i) {
+#pragma unroll 1
+        for (int j = 0; j < 64; ++j)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+    }
+    return false;
+}
+__device__ __forceinline__ bool wait_sleepy(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    for (uint32_t i = 0; i < ws::WAIT_POLLS / 4; ++i) {
+        if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
+        if (*abort_flag) return false;
     }
     return false;
 }
@@ -123,11 +138,11 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 const int st = jt & 1;
                 const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
                 const int j0 = jt * BC;
-                if (!wait_or_abort(bar(BAR_KE + st), ph ^ 1u, abort_flag)) { fail(1); break; }
+                if (!wait_sleepy(bar(BAR_KE + st), ph ^ 1u, abort_flag)) { fail(1); break; }
                 mbar_expect_tx(bar(BAR_KF + st), K_STAGE);
                 tma_load_3d(k_s + st * K_STAGE, &tmap_k, bar(BAR_KF + st), 0, j0, bh_kv);
                 tma_load_3d(k_s + st * K_STAGE + 16384, &tmap_k, bar(BAR_KF + st), 64, j0, bh_kv);
-                if (!wait_or_abort(bar(BAR_VE + st), ph ^ 1u, abort_flag)) { fail(2); break; }
+                if (!wait_sleepy(bar(BAR_VE + st), ph ^ 1u, abort_flag)) { fail(2); break; }
                 mbar_expect_tx(bar(BAR_VF + st), 2 * D * 128);
                 tma_load_3d(v_s + st * V_STAGE, &tmap_v, bar(BAR_VF + st), j0, 0, bh_kv);
                 tma_load_3d(v_s + st * V_STAGE + V_CHUNK, &tmap_v, bar(BAR_VF + st), j0 + 64, 0, bh_kv);
