@@ -46,6 +46,7 @@ typedef enum { HIFA4_F16 = 0, HIFA4_BF16 = 1, HIFA4_F32 = 2 } hifa4_dtype;
 enum { HIFA4_Q = 0, HIFA4_K = 1, HIFA4_V = 2 };               /* `which` */
 enum { HIFA4_PART_CODES = 0, HIFA4_PART_META = 1, HIFA4_PART_MMA = 2 }; /* `part` */
 enum { HIFA4_MAX_HEADS = 256, HIFA4_MAX_DEBUG_BLOCKS = 16 };
+#define HIFA4_STATIC_CALIB_MAX_FLOATS (1u << 20)   /* scratch limit of hifa4_smooth_calibrate_static */
 
 /* Problem shape.  Q is [B,Hq,N,d]; K and V are [B,Hkv,N,d] ("GQA and batch
  * handling", Appendix "Implementation Details").  d in {64,128,256};
@@ -142,6 +143,31 @@ int hifa4_smooth_calibrate(const void* q_cal, const void* k_cal, int S, int Hq, 
                            int Ncal, int d, const int* q_to_kv, int dt, int mode, float alpha,
                            float* s, float* inv_s, float* absmax_ws,
                            hifa4_calib_stats* host_stats, void* stream);
+
+/* hifa4_smooth_calibrate for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this entry point exists for deployment only.)
+ *   Who needs it: code that runs where cudaMalloc is off limits -- a serving process whose whole
+ *   device memory already belongs to an arena it may not grow, a plug-in called from a runtime
+ *   that forbids allocation on its worker threads, a latency-critical section that cannot take
+ *   the device-wide synchronization an allocation implies.  Such a caller still owns its inputs
+ *   and outputs (q_cal, k_cal, s, inv_s) but has nowhere to get the 2*S*Hkv*d-float scratch from.
+ *   What it does: the same computation, with the same kernels, as hifa4_smooth_calibrate; the
+ *   scratch is a fixed array of HIFA4_STATIC_CALIB_MAX_FLOATS floats (4 MiB) in device global
+ *   memory, which every GPU that loads this library holds until the process exits.  The call
+ *   makes no cudaMalloc/cudaFree and uses no allocating library routine.
+ *   Limits and rules:
+ *   - 2*S*Hkv*d must not exceed HIFA4_STATIC_CALIB_MAX_FLOATS, else HIFA4_ERR_WORKSPACE is
+ *     returned and nothing is enqueued (use hifa4_smooth_calibrate with your own workspace).
+ *   - The first call on each device looks up the device address of the array (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; each
+ *     call clears the part it uses before reducing into it.  Two calls whose kernels may overlap
+ *     on the GPU (different streams, no ordering between them) race on it: serialize them.
+ *   Arguments and results otherwise as hifa4_smooth_calibrate, minus absmax_ws. */
+int hifa4_smooth_calibrate_static(const void* q_cal, const void* k_cal, int S, int Hq, int Hkv,
+                                  int Ncal, int d, const int* q_to_kv, int dt, int mode,
+                                  float alpha, float* s, float* inv_s,
+                                  hifa4_calib_stats* host_stats, void* stream);
 
 /* Bytes of one buffer of hifa4_qkv for this shape; 0 on a bad argument. */
 size_t hifa4_quant_bytes(const hifa4_shape* shape, int which, int part);

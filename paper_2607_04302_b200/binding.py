@@ -85,6 +85,10 @@ def lib():
                                              C.c_int, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_float,
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(_CalibStats),
                                              C.c_void_p]
+        L.hifa4_smooth_calibrate_static.restype = C.c_int
+        L.hifa4_smooth_calibrate_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
+                                                    C.c_int, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_float,
+                                                    C.c_void_p, C.c_void_p, C.POINTER(_CalibStats), C.c_void_p]
         L.hifa4_quantize_qkv.restype = C.c_int
         L.hifa4_quantize_qkv.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.c_void_p, C.POINTER(_QKV), C.c_void_p, C.c_void_p]
@@ -99,7 +103,10 @@ def lib():
     return _lib
 
 
-EXPORTS = ("hifa4_status_string", "hifa4_get_counters", "hifa4_smooth_calibrate", "hifa4_quant_bytes",
+STATIC_CALIB_MAX_FLOATS = 1 << 20
+
+EXPORTS = ("hifa4_status_string", "hifa4_get_counters", "hifa4_smooth_calibrate",
+           "hifa4_smooth_calibrate_static", "hifa4_quant_bytes",
            "hifa4_quantize_qkv", "hifa4_attention_workspace_bytes", "hifa4_attention_fwd",
            "hifa4_attention_raw_workspace_bytes", "hifa4_attention_fwd_raw")
 
@@ -208,6 +215,27 @@ def smooth_calibrate(q_cal, k_cal, mode, alpha=0.0, q_to_kv=None):
                                       int(mode), float(alpha), _ptr(s), _ptr(inv_s), _ptr(ws),
                                       C.byref(stats), _stream())
     _check(rc, "hifa4_smooth_calibrate")
+    return s, inv_s
+
+
+def smooth_calibrate_static(q_cal, k_cal, mode, alpha=0.0, q_to_kv=None, s=None, inv_s=None):
+    """smooth_calibrate through the entry point that allocates nothing on the device: the scratch
+    is the library's fixed array (2*S*Hkv*d <= STATIC_CALIB_MAX_FLOATS, else Hifa4Error with status
+    3).  The caller may pass preallocated outputs s, inv_s [Hkv,d] float32; they are created here
+    only for convenience when omitted (the C entry point itself never allocates)."""
+    assert q_cal.is_cuda and k_cal.is_cuda and q_cal.is_contiguous() and k_cal.is_contiguous()
+    S, Hq, Ncal, d = q_cal.shape
+    Hkv = k_cal.shape[1]
+    if s is None:
+        s = torch.empty((Hkv, d), dtype=torch.float32, device=q_cal.device)
+    if inv_s is None:
+        inv_s = torch.empty_like(s)
+    keep, mp = _map_arr(q_to_kv)
+    stats = _CalibStats()
+    rc = lib().hifa4_smooth_calibrate_static(_ptr(q_cal), _ptr(k_cal), S, Hq, Hkv, Ncal, d, mp,
+                                             _DT[q_cal.dtype], int(mode), float(alpha), _ptr(s), _ptr(inv_s),
+                                             C.byref(stats), _stream())
+    _check(rc, "hifa4_smooth_calibrate_static")
     return s, inv_s
 
 
