@@ -157,66 +157,82 @@ __device__ __forceinline__ float p_of_score(float acc, float c1, float mL)
 //   need = max(bits(At) - bits(1.75 S) - 1 + 2^23, 0) >> 23   (0, 1 or 2)
 // and the pair rule "level-2 bit = 1 iff max(need) = 2 or min(need) >= 1" is a = (n0 + n1 + 2) >> 2,
 // k = max(need, a).  Multiplications, additions and FMAs run two elements at a time (f32x2).
-template <int NU, bool DBG>
-__device__ __forceinline__ void exp_quantize_units(const float (&acc)[NU * 8], float c1, float mL, float A,
-                                                   uint32_t (&w)[NU * 4], uint8_t* dump_codes, float* dump_step)
+struct PQuantConst {              // per (row, 64-key group, tile) constants of the fused quantizer
+    uint64_t c1c1, nml, inv44, s44;
+    uint32_t c0_bits, s4_bits;
+    int tadd;
+};
+
+// Constants from the group maximum A of P.  A = 0 (every key masked) needs no branch: the scale
+// code clamps to 0, every p is 0 and every product below is an exact zero.
+__device__ __forceinline__ PQuantConst p_quant_const(float c1, float mL, float A)
 {
-    if (A == 0.f) {
-#pragma unroll
-        for (int i = 0; i < NU * 4; ++i) w[i] = 0u;
-        if (DBG) {
-            if (dump_codes) {
-#pragma unroll
-                for (int i = 0; i < NU / 2; ++i) reinterpret_cast<uint4*>(dump_codes)[i] = make_uint4(0, 0, 0, 0);
-            }
-            if (dump_step) {
-#pragma unroll
-                for (int i = 0; i < NU / 2; ++i) reinterpret_cast<float4*>(dump_step)[i] = make_float4(0, 0, 0, 0);
-            }
-        }
-        return;
-    }
+    PQuantConst k;
     const int code = e6m2_code_for_max(A);
     const float S = e6m2_value(code);
     const float inv4 = e6m2_inv4(code);
     const float S4 = __uint_as_float(__float_as_uint(S) - (2u << 23));     // S / 4
-    const int tadd = (1 << 23) - ((int)__float_as_uint(1.75f * S) + 1);
-    const uint32_t MAGIC_BITS = 0x4B400000u;                               // 1.5 * 2^23
-    const uint32_t c0_bits = __float_as_uint(-12582912.f * S4);            // -magic * S/4 at shift 0
-    const uint64_t c1c1 = pack2(c1, c1), nml = pack2(-mL, -mL);
-    const uint64_t inv44 = pack2(inv4, inv4), s44 = pack2(S4, S4);
+    k.tadd = (1 << 23) - ((int)__float_as_uint(1.75f * S) + 1);
+    k.c0_bits = __float_as_uint(-12582912.f * S4);                         // -1.5 * 2^23 * S/4
+    k.s4_bits = __float_as_uint(S4);
+    k.c1c1 = pack2(c1, c1);
+    k.nml = pack2(-mL, -mL);
+    k.inv44 = pack2(inv4, inv4);
+    k.s44 = pack2(S4, S4);
+    return k;
+}
+
+// P = exp2(acc * c1 - mL) rounded to FP16 for the 8 keys of unit u.
+template <int NU>
+__device__ __forceinline__ void exp_unit(const float (&acc)[NU * 8], int u, const PQuantConst& k, float (&p)[8])
+{
 #pragma unroll
-    for (int u = 0; u < NU; ++u) {
+    for (int i = 0; i < 8; i += 2) {
+        float t0, t1;
+        unpack2(fma2(pack2(acc[8 * u + i], acc[8 * u + i + 1]), k.c1c1, k.nml), t0, t1);
+        exp2_f16_pair(t0, t1, p[i], p[i + 1]);
+    }
+}
+
+// Units U0..U1-1 of a thread's NU units: acc -> P (FP16) -> P-hat image words w[4u..4u+3].
+// The exponentials of unit u+1 are issued before unit u is quantized, so that the MUFU latency of
+// one unit hides behind the ALU/FMA work of the previous one.
+template <int NU, int U0, int U1, bool DBG>
+__device__ __forceinline__ void exp_quantize_units(const float (&acc)[NU * 8], const PQuantConst& k, bool zero_group,
+                                                   uint32_t (&w)[NU * 4], uint8_t* dump_codes, float* dump_step)
+{
+    const uint32_t MAGIC_BITS = 0x4B400000u;                               // 1.5 * 2^23
+    float pn[8];
+    exp_unit<NU>(acc, U0, k, pn);
+#pragma unroll
+    for (int u = U0; u < U1; ++u) {
         float p[8];
 #pragma unroll
-        for (int i = 0; i < 8; i += 2) {
-            float t0, t1;
-            unpack2(fma2(pack2(acc[8 * u + i], acc[8 * u + i + 1]), c1c1, nml), t0, t1);
-            exp2_f16_pair(t0, t1, p[i], p[i + 1]);
-        }
+        for (int i = 0; i < 8; ++i) p[i] = pn[i];
+        if (u + 1 < U1) exp_unit<NU>(acc, u + 1, k, pn);
         const float At0 = fmaxf(max3(p[0], p[1], p[2]), p[3]);
         const float At1 = fmaxf(max3(p[4], p[5], p[6]), p[7]);
-        const int n0 = max((int)__float_as_uint(At0) + tadd, 0) >> 23;
-        const int n1 = max((int)__float_as_uint(At1) + tadd, 0) >> 23;
+        const int n0 = max((int)__float_as_uint(At0) + k.tadd, 0) >> 23;
+        const int n1 = max((int)__float_as_uint(At1) + k.tadd, 0) >> 23;
         const int a = (n0 + n1 + 2) >> 2;
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
             const uint32_t ks = (uint32_t)max(h ? n1 : n0, a) << 23;
             const float magic = __uint_as_float(MAGIC_BITS + ks);
-            const float ck = __uint_as_float(c0_bits + ks);
+            const float ck = __uint_as_float(k.c0_bits + ks);
             const uint64_t mm = pack2(magic, magic), cc = pack2(ck, ck);
             float v0, v1, v2, v3;
-            const uint64_t y01 = add2(mul2_rz(pack2(p[4 * h], p[4 * h + 1]), inv44), mm);
-            const uint64_t y23 = add2(mul2_rz(pack2(p[4 * h + 2], p[4 * h + 3]), inv44), mm);
-            unpack2(fma2(y01, s44, cc), v0, v1);
-            unpack2(fma2(y23, s44, cc), v2, v3);
+            const uint64_t y01 = add2(mul2_rz(pack2(p[4 * h], p[4 * h + 1]), k.inv44), mm);
+            const uint64_t y23 = add2(mul2_rz(pack2(p[4 * h + 2], p[4 * h + 3]), k.inv44), mm);
+            unpack2(fma2(y01, k.s44, cc), v0, v1);
+            unpack2(fma2(y23, k.s44, cc), v2, v3);
             asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h]) : "f"(v1), "f"(v0));
             asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h + 1]) : "f"(v3), "f"(v2));
             if (DBG) {
                 float y0, y1, y2, y3;
                 unpack2(y01, y0, y1);
                 unpack2(y23, y2, y3);
-                if (dump_step) dump_step[2 * u + h] = __uint_as_float(__float_as_uint(S4) + ks);
+                if (dump_step) dump_step[2 * u + h] = zero_group ? 0.f : __uint_as_float(k.s4_bits + ks);
                 if (dump_codes)
                     reinterpret_cast<uint32_t*>(dump_codes)[2 * u + h] =
                         (__float_as_uint(y0) & 15u) | ((__float_as_uint(y1) & 15u) << 8) |

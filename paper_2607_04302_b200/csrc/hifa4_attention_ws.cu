@@ -299,7 +299,8 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             }
             {
                 uint32_t w[NU * 4];
-                exp_quantize_units<NU, DBG>(p, args.c1, mL, A, w, dc, ds);
+                const PQuantConst qc = p_quant_const(args.c1, mL, A);
+                exp_quantize_units<NU, 0, NU, DBG>(p, qc, A == 0.f, w, dc, ds);
                 if constexpr (KS == 2) tmem_st32(t_s + kq * (KPT / 2), w);
                 else tmem_st16(t_s + kq * (KPT / 2), w);
             }
