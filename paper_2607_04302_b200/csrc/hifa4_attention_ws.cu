@@ -150,46 +150,55 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         }
     } else if (warp == W_MMA) {
         // ------------------------------------------------------------------ tcgen05 issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc_s = umma_idesc_bf16(128, BC);
-            constexpr uint32_t idesc_o = umma_idesc_bf16(128, O_COLS);
-            const uint32_t k_lo = umma_desc_lo(k_s), v_lo = umma_desc_lo(v_s);
-            auto issue_qk = [&](int jt) {                 // S(jt) -> buffer jt % 2 from K stage jt % 2
-                const int st = jt & 1;
-                const uint32_t d = tmem + S_COL + st * 128;
-                const uint32_t b0 = k_lo + st * (K_STAGE >> 4);
+        // The whole warp runs the loop and the waits (warp-uniform control flow keeps the operand
+        // arithmetic cheap); one elected lane issues the MMAs and the commits.
+        constexpr uint32_t idesc_s = umma_idesc_bf16(128, BC);
+        constexpr uint32_t idesc_o = umma_idesc_bf16(128, O_COLS);
+        const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+        const uint32_t k_lo = umma_desc_lo(k_s), v_lo = umma_desc_lo(v_s);
+        const bool leader = elect_one();
+        auto issue_qk = [&](int jt) {                 // S(jt) -> buffer jt % 2 from K stage jt % 2
+            const int st = jt & 1;
+            const uint32_t d = tm + S_COL + st * 128;
+            const uint32_t b0 = k_lo + st * (K_STAGE >> 4);
+            if (leader) {
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)               // 16 channels per step = 8 columns of the Q image
-                    umma_bf16_ts_lo(d, tmem + QT_COL + kk * 8, b0 + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2, idesc_s,
+                    umma_bf16_ts_lo(d, tm + QT_COL + kk * 8, b0 + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2, idesc_s,
                                     kk ? 1u : 0u);
                 umma_commit(bar(BAR_SF + st));
                 umma_commit(bar(BAR_KE + st));
-            };
-            bool ok = wait_or_abort(bar(BAR_QT), 0, abort_flag);
-            for (int jt = 0; ok && jt < min(2, n_tiles); ++jt) {
-                ok = wait_or_abort(bar(BAR_KF + jt), 0, abort_flag);
-                if (ok) { tc_fence_after(); issue_qk(jt); }
             }
-            if (!ok) fail(3);
-            for (int jt = 0; ok && jt < n_tiles; ++jt) {
-                const int st = jt & 1;
-                const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
-                if (!wait_or_abort(bar(BAR_VF + st), ph, abort_flag)) { fail(6); break; }
-                if (!wait_or_abort(bar(BAR_PF + st), ph, abort_flag)) { fail(7); break; }
-                tc_fence_after();
-                const uint32_t a0 = tmem + S_COL + st * 128;
-                const uint32_t b0 = v_lo + st * (V_STAGE >> 4);
+            __syncwarp();
+        };
+        bool ok = wait_or_abort(bar(BAR_QT), 0, abort_flag);
+        for (int jt = 0; ok && jt < min(2, n_tiles); ++jt) {
+            ok = wait_or_abort(bar(BAR_KF + jt), 0, abort_flag);
+            if (ok) { tc_fence_after(); issue_qk(jt); }
+        }
+        if (!ok && leader) fail(3);
+        for (int jt = 0; ok && jt < n_tiles; ++jt) {
+            const int st = jt & 1;
+            const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
+            if (!wait_or_abort(bar(BAR_VF + st), ph, abort_flag)) { if (leader) fail(6); break; }
+            if (!wait_or_abort(bar(BAR_PF + st), ph, abort_flag)) { if (leader) fail(7); break; }
+            tc_fence_after();
+            const uint32_t a0 = tm + S_COL + st * 128;
+            const uint32_t b0 = v_lo + st * (V_STAGE >> 4);
+            const uint32_t acc0 = jt > 0 ? 1u : 0u;
+            if (leader) {
 #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)          // 16 keys per step = 8 columns of packed BF16 pairs
-                    umma_bf16_ts_lo(tmem, a0 + kk * 8, b0 + (kk >> 2) * (V_CHUNK >> 4) + (kk & 3) * 2, idesc_o,
-                                    (jt > 0 || kk > 0) ? 1u : 0u);
+                    umma_bf16_ts_lo(tm, a0 + kk * 8, b0 + (kk >> 2) * (V_CHUNK >> 4) + (kk & 3) * 2, idesc_o,
+                                    kk ? 1u : acc0);
                 umma_commit(bar(BAR_PV));
                 umma_commit(bar(BAR_VE + st));
-                if (jt + 2 < n_tiles) {
-                    if (!wait_or_abort(bar(BAR_KF + st), (uint32_t)((jt + 2) >> 1) & 1u, abort_flag)) { fail(4); break; }
-                    tc_fence_after();
-                    issue_qk(jt + 2);
-                }
+            }
+            __syncwarp();
+            if (jt + 2 < n_tiles) {
+                if (!wait_or_abort(bar(BAR_KF + st), (uint32_t)((jt + 2) >> 1) & 1u, abort_flag)) { if (leader) fail(4); break; }
+                tc_fence_after();
+                issue_qk(jt + 2);
             }
         }
     } else {
