@@ -46,18 +46,23 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while the GPU is under load.
+
+    nvidia-smi needs ~100 ms per sample, so a short timed region yields few samples; the sampler is
+    started before warm-up and the benchmark keeps the GPU busy (same step function) until at least
+    a few samples fall inside the marked window."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.index, self.rows, self.proc, self.thr = index, [], None, None
+        self.t0 = self.t1 = None
 
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             return
@@ -66,7 +71,19 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            self.rows.append((time.perf_counter(), [c.strip() for c in line.split(",")]))
+
+    def mark_begin(self):
+        self.t0 = time.perf_counter()
+
+    def mark_end(self):
+        self.t1 = time.perf_counter()
+
+    def samples_in_window(self):
+        if self.t0 is None:
+            return 0
+        t1 = self.t1 if self.t1 is not None else time.perf_counter()
+        return sum(1 for t, _ in self.rows if self.t0 <= t <= t1)
 
     def stop(self):
         if self.proc is None:
@@ -76,19 +93,22 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], None, set()
+        sm, mx, reasons, power = [], None, set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for t, r in self.rows:
+            if self.t0 is None or not (self.t0 <= t <= (self.t1 or t)):
+                continue
             try:
-                sm.append(float(r[0])); mx = float(r[1])
+                sm.append(float(r[0])); mx = float(r[1]); power.append(float(r[2]))
             except (ValueError, IndexError):
                 continue
             for n, v in zip(names, r[4:8]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
-        busy = sorted(sm)[len(sm) // 2:] if sm else []          # upper half = samples under load
-        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": mx,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx,
+                "reasons": sorted(reasons), "samples": len(sm),
+                "power_w_max": max(power) if power else None,
+                "window": "timed steps plus identical untimed steps run until 8 samples were taken"}
 
 
 def oracle_time(cfg, q, k, v, s, inv_s, heads):
@@ -159,8 +179,8 @@ def run_reference(args, cfg, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="C2", help="C2 (headline), C3, C4, C5 or C5@<N>")
     ap.add_argument("--noncausal", action="store_true")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -227,17 +247,18 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(args.warmup):
         flush.zero_()
         step()
     barrier()
     assert int(status.item()) == 0, f"device status {int(status.item())}"
 
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     c0 = hb.get_counters()["launches"]
     ev = []
     barrier()
+    sampler.mark_begin()
     for _ in range(args.steps):
         flush.zero_()                                                   # L2 flush, outside the events
         a = torch.cuda.Event(enable_timing=True)
@@ -248,6 +269,14 @@ def main():
         ev.append((a, mid, b))
     barrier()
     launches = hb.get_counters()["launches"] - c0
+    # keep the same load on the GPU (untimed) until nvidia-smi has taken a few samples of it
+    t_lim = time.perf_counter() + 3.0
+    while sampler.proc is not None and sampler.samples_in_window() < 8 and time.perf_counter() < t_lim:
+        for _ in range(20):
+            flush.zero_()
+            step()
+        torch.cuda.synchronize()
+    sampler.mark_end()
     clocks = sampler.stop()
     step_ms = [a.elapsed_time(b) for a, _, b in ev]
     attn_ms = [m.elapsed_time(b) for _, m, b in ev]
