@@ -90,8 +90,12 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int N = args.N;
     const int n_qt = (N + 127) / 128;
-    const int qt = n_qt - 1 - (int)blockIdx.x;              // heaviest causal tiles are scheduled first
-    const int h = blockIdx.y, b = blockIdx.z;
+    // 1-D grid, query block outermost and descending: with a causal mask the work of a CTA grows with
+    // its query block, so every heaviest CTA (all heads, all batches) is scheduled before any lighter one
+    const int n_bh = args.B * args.Hq;
+    const int qt = n_qt - 1 - (int)(blockIdx.x / n_bh);
+    const int bh = (int)(blockIdx.x % n_bh);
+    const int h = bh % args.Hq, b = bh / args.Hq;
     const int g = args.map.kv_of[h];
     const int q0 = qt * 128;
     const int bh_q = b * args.Hq + h, bh_kv = b * args.Hkv + g;
@@ -420,7 +424,7 @@ static int launch_ws(const hifa4_shape& sh, const CUtensorMap& mq, const CUtenso
             return HIFA4_ERR_CUDA;
         attr_set = true;
     }
-    dim3 grid((sh.N + 127) / 128, sh.Hq, sh.B);
+    dim3 grid((unsigned)(((sh.N + 127) / 128) * sh.Hq * sh.B));
     kern<<<grid, (4 * KS + 2) * 32, ws::SMEM_BYTES, st>>>(mq, mk, mv, args);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? HIFA4_OK : HIFA4_ERR_CUDA;
