@@ -211,7 +211,6 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         const int r_loc = quarter * 32 + lane;                    // row inside the tile = TMEM lane
         const int row = q0 + r_loc;
         const uint32_t t_lane = tmem + ((uint32_t)(quarter * 32) << 16);
-        const uint32_t xbar = bar(BAR_X + quarter);
         const float LOG2E = 1.4426950408889634f;
         const int key_lim = args.causal ? min(row, N - 1) : N - 1;
         int dbg_slot = -1;
@@ -244,33 +243,35 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             if (lane == 0) mbar_arrive(bar(BAR_QT));
         } else { fail(13); ok = false; }
 
-        for (int jt = 0; ok && jt < n_tiles; ++jt) {
+        // The KS warps of a row quarter meet once per tile at a hardware named barrier (their partial
+        // maxima go through shared memory).  It cannot time out, so every warp executes it exactly
+        // n_tiles times: after a failed wait a warp keeps looping and only takes the barrier.
+        for (int jt = 0; jt < n_tiles; ++jt) {
             const int j0 = jt * BC;
             const uint32_t par = (uint32_t)jt & 1u;
             const int sb = jt & 1;                             // S / P-hat buffer and its barrier pair
             const uint32_t ph2 = (uint32_t)(jt >> 1) & 1u;
             const uint32_t t_s = t_lane + S_COL + sb * 128;
-            if (!wait_or_abort(bar(BAR_SF + sb), ph2, abort_flag)) { fail(8); ok = false; break; }
-            tc_fence_after();
-            float p[KPT];
-#pragma unroll
-            for (int cc = 0; cc < KPT / 32; ++cc) {
-                uint32_t r[32];
-                tmem_ld32(t_s + kq * KPT + cc * 32, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) p[cc * 32 + i] = __uint_as_float(r[i]);
-            }
-
-            // row maximum over the 128-key tile (line 7): own keys, then the other splits'
-            const bool need_mask = (args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N);
             const int kbase = j0 + kq * KPT;
-            if (need_mask) {                                   // masked scores become -inf: exp gives exact zeros
+            float p[KPT];
+            float mx = -INFINITY;
+            if (ok && !wait_or_abort(bar(BAR_SF + sb), ph2, abort_flag)) { fail(8); ok = false; }
+            if (ok) {
+                tc_fence_after();
 #pragma unroll
-                for (int i = 0; i < KPT; ++i) p[i] = (kbase + i > key_lim) ? -INFINITY : p[i];
-            }
-            float mx;
-            {
+                for (int cc = 0; cc < KPT / 32; ++cc) {
+                    uint32_t r[32];
+                    tmem_ld32(t_s + kq * KPT + cc * 32, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) p[cc * 32 + i] = __uint_as_float(r[i]);
+                }
+                // row maximum over the 128-key tile (line 7): own keys, then the other splits'
+                const bool need_mask = (args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N);
+                if (need_mask) {                               // masked scores become -inf: exp gives exact zeros
+#pragma unroll
+                    for (int i = 0; i < KPT; ++i) p[i] = (kbase + i > key_lim) ? -INFINITY : p[i];
+                }
                 float t4[KPT / 4];
 #pragma unroll
                 for (int i = 0; i < KPT / 4; ++i) t4[i] = fmaxf(max3(p[4 * i], p[4 * i + 1], p[4 * i + 2]), p[4 * i + 3]);
@@ -279,14 +280,13 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
 #pragma unroll
                     for (int i = 0; i < w; ++i) t4[i] = fmaxf(t4[i], t4[i + w]);
                 mx = t4[0];
+                xmax[(par * 4 + kq) * 128 + r_loc] = mx;
+                tc_fence_before();                             // S(jt) is in registers: others may overwrite it with P-hat
             }
-            float gmax = mx;                                   // maximum over this thread's 64-key group
-            xmax[(par * 4 + kq) * 128 + r_loc] = mx;
-            tc_fence_before();                                 // S(jt) is in registers: others may overwrite it with P-hat
-            __syncwarp();
-            if (lane == 0) mbar_arrive(xbar);
-            if (!wait_or_abort(xbar, par, abort_flag)) { fail(9); ok = false; break; }
+            named_bar_sync(1 + quarter, 32 * KS);
+            if (!ok) continue;
             tc_fence_after();
+            float gmax = mx;                                   // maximum over this thread's 64-key group
 #pragma unroll
             for (int o = 1; o < KS; ++o) {
                 const float other = xmax[(par * 4 + (kq ^ o)) * 128 + r_loc];
@@ -322,7 +322,7 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             // Every warp observes every phase of the PV barrier, in order: a parity wait can only tell
             // the last two phases apart, so skipping one would alias.
             if (jt > 0) {
-                if (!wait_or_abort(bar(BAR_PV), par ^ 1u, abort_flag)) { fail(10); ok = false; break; }
+                if (!wait_or_abort(bar(BAR_PV), par ^ 1u, abort_flag)) { fail(10); ok = false; continue; }
                 tc_fence_after();
             }
             if (__any_sync(0xffffffffu, rsc != 1.f)) {

@@ -204,6 +204,12 @@ __device__ __forceinline__ void umma_bf16_ts_lo(uint32_t d_tmem, uint32_t a_tmem
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(UMMA_DESC_HI_SW128), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Hardware named barrier among `nthreads` threads of the CTA (whole warps).  It has no time-out:
+// every participant must reach it the same number of times on every path, failure paths included.
+__device__ __forceinline__ void named_bar_sync(uint32_t id, uint32_t nthreads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
 // One lane of a converged warp (the same lane every time while the warp stays converged).
 __device__ __forceinline__ bool elect_one()
 {
