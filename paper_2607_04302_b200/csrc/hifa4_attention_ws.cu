@@ -36,7 +36,7 @@ constexpr int XCHG_BYTES = 2 * 4 * 128 * 4;
 constexpr int SMEM_BYTES = XCHG_OFF + XCHG_BYTES + 1024;
 constexpr int O_COLS = D + 16, QT_COL = 144, S_COL = 256, TMEM_COLS = 512;
 enum { BAR_Q = 0, BAR_KF = 1, BAR_KE = 3, BAR_VF = 5, BAR_VE = 7, BAR_SF = 9, BAR_PF = 11,
-       BAR_PV = 13, BAR_X = 14, BAR_QT = 18, N_BARS = 19 };
+       BAR_PV = 13, BAR_X = 14, BAR_QT = 22, N_BARS = 23 };
 constexpr uint32_t WAIT_POLLS = 1u << 20;           // each poll blocks for a hardware-defined slice
 }  // namespace ws
 
@@ -111,7 +111,7 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             mbar_init(bar(BAR_SF + s), 1); mbar_init(bar(BAR_PF + s), NSW);
         }
         mbar_init(bar(BAR_PV), 1); mbar_init(bar(BAR_QT), NSW);
-        for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_X + i), KS);
+        for (int i = 0; i < 8; ++i) mbar_init(bar(BAR_X + i), KS);
         fence_barrier_init();
     }
     if (warp == W_MMA) { tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS); tmem_relinquish(); }
@@ -243,10 +243,47 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             if (lane == 0) mbar_arrive(bar(BAR_QT));
         } else { fail(13); ok = false; }
 
-        // The KS warps of a row quarter meet once per tile at a hardware named barrier (their partial
-        // maxima go through shared memory).  It cannot time out, so every warp executes it exactly
-        // n_tiles times: after a failed wait a warp keeps looping and only takes the barrier.
-        for (int jt = 0; jt < n_tiles; ++jt) {
+        // The scores of tile jt+1 are pulled into registers, reduced and published while tile jt is
+        // still being quantized (S is double-buffered), so the row-maximum exchange of a tile is usually
+        // complete by the time its turn comes and the KS warps of a row quarter need not run in phase.
+        auto fetch_scores = [&](int jt, float (&sc)[KPT]) -> float {
+            const int j0 = jt * BC, kb = j0 + kq * KPT;
+            const uint32_t t_src = t_lane + S_COL + (jt & 1) * 128 + kq * KPT;
+#pragma unroll
+            for (int cc = 0; cc < KPT / 32; ++cc) {
+                uint32_t r[32];
+                tmem_ld32(t_src + cc * 32, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) sc[cc * 32 + i] = __uint_as_float(r[i]);
+            }
+            const bool need_mask = (args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N);
+            if (need_mask) {                                   // masked scores become -inf: exp gives exact zeros
+#pragma unroll
+                for (int i = 0; i < KPT; ++i) sc[i] = (kb + i > key_lim) ? -INFINITY : sc[i];
+            }
+            float t4[KPT / 4];
+#pragma unroll
+            for (int i = 0; i < KPT / 4; ++i) t4[i] = fmaxf(max3(sc[4 * i], sc[4 * i + 1], sc[4 * i + 2]), sc[4 * i + 3]);
+#pragma unroll
+            for (int w = KPT / 8; w >= 1; w >>= 1)
+#pragma unroll
+                for (int i = 0; i < w; ++i) t4[i] = fmaxf(t4[i], t4[i + w]);
+            xmax[((jt & 1) * 4 + kq) * 128 + r_loc] = t4[0];
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_X + quarter * 2 + (jt & 1)));
+            return t4[0];
+        };
+
+        float pn[KPT];                                        // scores of the next tile
+        float mx_next = -INFINITY;
+        if (ok) {
+            if (wait_or_abort(bar(BAR_SF), 0, abort_flag)) { tc_fence_after(); mx_next = fetch_scores(0, pn); }
+            else { fail(8); ok = false; }
+        }
+
+        for (int jt = 0; ok && jt < n_tiles; ++jt) {
             const int j0 = jt * BC;
             const uint32_t par = (uint32_t)jt & 1u;
             const int sb = jt & 1;                             // S / P-hat buffer and its barrier pair
@@ -254,39 +291,12 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             const uint32_t t_s = t_lane + S_COL + sb * 128;
             const int kbase = j0 + kq * KPT;
             float p[KPT];
-            float mx = -INFINITY;
-            if (ok && !wait_or_abort(bar(BAR_SF + sb), ph2, abort_flag)) { fail(8); ok = false; }
-            if (ok) {
-                tc_fence_after();
 #pragma unroll
-                for (int cc = 0; cc < KPT / 32; ++cc) {
-                    uint32_t r[32];
-                    tmem_ld32(t_s + kq * KPT + cc * 32, r);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) p[cc * 32 + i] = __uint_as_float(r[i]);
-                }
-                // row maximum over the 128-key tile (line 7): own keys, then the other splits'
-                const bool need_mask = (args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N);
-                if (need_mask) {                               // masked scores become -inf: exp gives exact zeros
-#pragma unroll
-                    for (int i = 0; i < KPT; ++i) p[i] = (kbase + i > key_lim) ? -INFINITY : p[i];
-                }
-                float t4[KPT / 4];
-#pragma unroll
-                for (int i = 0; i < KPT / 4; ++i) t4[i] = fmaxf(max3(p[4 * i], p[4 * i + 1], p[4 * i + 2]), p[4 * i + 3]);
-#pragma unroll
-                for (int w = KPT / 8; w >= 1; w >>= 1)
-#pragma unroll
-                    for (int i = 0; i < w; ++i) t4[i] = fmaxf(t4[i], t4[i + w]);
-                mx = t4[0];
-                xmax[(par * 4 + kq) * 128 + r_loc] = mx;
-                tc_fence_before();                             // S(jt) is in registers: others may overwrite it with P-hat
-            }
-            named_bar_sync(1 + quarter, 32 * KS);
-            if (!ok) continue;
+            for (int i = 0; i < KPT; ++i) p[i] = pn[i];
+            float mx = mx_next, gmax = mx_next;                // gmax: maximum over this thread's 64-key group
+            // row maximum over the 128-key tile (line 7): own keys, then the other splits'
+            if (!wait_or_abort(bar(BAR_X + quarter * 2 + sb), ph2, abort_flag)) { fail(9); ok = false; break; }
             tc_fence_after();
-            float gmax = mx;                                   // maximum over this thread's 64-key group
 #pragma unroll
             for (int o = 1; o < KS; ++o) {
                 const float other = xmax[(par * 4 + (kq ^ o)) * 128 + r_loc];
@@ -313,7 +323,14 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             {
                 uint32_t w[NU * 4];
                 const PQuantConst qc = p_quant_const(args.c1, mL, A);
-                exp_quantize_units<NU, 0, NU, DBG>(p, qc, A == 0.f, w, dc, ds);
+                constexpr int U_SPLIT = (3 * NU) / 4;
+                exp_quantize_units<NU, 0, U_SPLIT, DBG>(p, qc, A == 0.f, w, dc, ds);
+                if (jt + 1 < n_tiles) {                        // next tile's scores and partial maximum
+                    if (!wait_or_abort(bar(BAR_SF + (sb ^ 1)), (uint32_t)((jt + 1) >> 1) & 1u, abort_flag)) { fail(8); ok = false; break; }
+                    tc_fence_after();
+                    mx_next = fetch_scores(jt + 1, pn);
+                }
+                exp_quantize_units<NU, U_SPLIT, NU, DBG>(p, qc, A == 0.f, w, dc, ds);
                 if constexpr (KS == 2) tmem_st32(t_s + kq * (KPT / 2), w);
                 else tmem_st16(t_s + kq * (KPT / 2), w);
             }
@@ -322,7 +339,7 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             // Every warp observes every phase of the PV barrier, in order: a parity wait can only tell
             // the last two phases apart, so skipping one would alias.
             if (jt > 0) {
-                if (!wait_or_abort(bar(BAR_PV), par ^ 1u, abort_flag)) { fail(10); ok = false; continue; }
+                if (!wait_or_abort(bar(BAR_PV), par ^ 1u, abort_flag)) { fail(10); ok = false; break; }
                 tc_fence_after();
             }
             if (__any_sync(0xffffffffu, rsc != 1.f)) {
