@@ -114,6 +114,20 @@ class ClockSampler:
                 "window": "timed steps plus identical untimed steps run until 8 samples were taken"}
 
 
+def max_over_ranks(dist, ms: float, device) -> float:
+    """Device time of the slowest rank (the job is as slow as its slowest rank)."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(cfg, world: int, steps: int, total_ms: float) -> float:
+    """Aggregate over all ranks: every rank processes its own copy of the workload (weak scaling)."""
+    return world * attn_flops(cfg) * steps / (total_ms * 1e-3) / 1e12
+
+
 def oracle_time(cfg, q, k, v, s, inv_s, heads):
     """Time the CPU oracle, as it stands, on whole heads of the workload (batch 0)."""
     from oracle import hifa4_oracle as orc
@@ -285,10 +299,7 @@ def main():
     attn_ms = [m.elapsed_time(b) for _, m, b in ev]
     quant_ms = [a.elapsed_time(m) for a, m, _ in ev]
     total_ms = sum(step_ms)
-    if dist is not None:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(dist, total_ms, dev)
     assert int(status.item()) == 0, f"device status {int(status.item())}"
 
     # ---- end to end through the raw C-ABI entry point with host buffers (pinned), copies timed
@@ -316,12 +327,9 @@ def main():
         b.record()
         barrier()
         e_ms = a.elapsed_time(b)
-        if dist is not None:
-            t = torch.tensor([e_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_ms = max_over_ranks(dist, e_ms, dev)
         h2d = (pq.numel() + pk.numel() + pv.numel()) * pq.element_size()
-        e2e = {"value": world * attn_flops(cfg) * n_e2e / (e_ms * 1e-3) / 1e12, "unit": UNIT,
+        e2e = {"value": whole_job_tflops(cfg, world, n_e2e, e_ms), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": po.numel() * 4, "ms_per_step": e_ms / n_e2e}
 
     if rank != 0:
@@ -331,7 +339,7 @@ def main():
 
     peaks = measured_peaks()
     fl = attn_flops(cfg)
-    value = world * fl * args.steps / (total_ms * 1e-3) / 1e12
+    value = whole_job_tflops(cfg, world, args.steps, total_ms)
     attn_avg_ms = sum(attn_ms) / len(attn_ms)
     achieved = fl / (attn_avg_ms * 1e-3) / 1e12
     roofline = {"bound": "tensor", "kernel": "attention_fwd_kernel", "achieved": achieved, "peak": peaks["bf16"],

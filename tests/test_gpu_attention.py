@@ -118,3 +118,37 @@ def test_sweep_point_sampled(hb, par, causal):
     blocks = [(0, 0, 0), (3, 31, 15), (1, 17, 7)]
     res = par.run_case(cfg, DEV, blocks=blocks, check_quant=False, rows_per_block=16)
     print(par.assert_within_bars(res, f"C5 N=2048 causal={causal}"))
+
+
+def test_sweep_point_8k_sampled(hb, par):
+    """Configuration 5 at N = 8192 (B = 4, causal): 8192 work items on the persistent kernel."""
+    cfg = synth.config("C5", N=8192, cal_samples=2, cal_tokens=256)
+    blocks = [(0, 0, 0), (3, 31, 63), (2, 9, 31), (1, 30, 1)]
+    res = par.run_case(cfg, DEV, blocks=blocks, check_quant=False, rows_per_block=12)
+    print(par.assert_within_bars(res, "C5 N=8192 causal"))
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_largest_sequence_properties(hb, causal):
+    """N = 32768 (the top of the sequence sweep), too large for the oracle: properties that hold at any
+    size.  With V constant per channel the output must be that constant's HIF4 value times
+    rowsum(P-hat) / FP16(rowsum(P-hat)): numerator and normalizer come from the same P-hat
+    (P-Reordering through the ones column), whatever the scores are.  Reruns are bit-identical."""
+    B, Hq, Hkv, N, d = 1, 4, 2, 32768, 128
+    gen = torch.Generator(device=DEV).manual_seed(7)
+    q = torch.randn((B, Hq, N, d), generator=gen, device=DEV).to(torch.bfloat16)
+    k = torch.randn((B, Hkv, N, d), generator=gen, device=DEV).to(torch.bfloat16)
+    consts = torch.linspace(-3.0, 3.0, d, device=DEV).to(torch.bfloat16)
+    v = consts.expand(B, Hkv, N, d).contiguous()
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    qkv = hb.quantize_qkv(q, k, v, d_status=status)
+    out = hb.attention_fwd(qkv, causal, Bc=128, d_status=status)
+    out2 = hb.attention_fwd(qkv, causal, Bc=128, d_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(out, out2) and torch.isfinite(out).all()
+    vhat = qkv.v_mma[0, 0, :, 0].float()                       # V-hat of each channel (constant along tokens)
+    assert torch.equal(qkv.v_mma[0, 0], vhat[:, None].expand(d, N).to(torch.bfloat16))
+    rel = (out / vhat[None, None, None, :].clamp_min(-1e30) - 1.0)
+    rel = rel[..., vhat != 0]
+    assert rel.abs().max().item() <= 2.0 ** -10                # only the FP16 rounding of the normalizer is left
