@@ -44,7 +44,7 @@ typedef enum {
 typedef enum { HIFA4_F16 = 0, HIFA4_BF16 = 1, HIFA4_F32 = 2 } hifa4_dtype;
 
 enum { HIFA4_Q = 0, HIFA4_K = 1, HIFA4_V = 2 };               /* `which` */
-enum { HIFA4_PART_CODES = 0, HIFA4_PART_META = 1, HIFA4_PART_MMA = 2 }; /* `part` */
+enum { HIFA4_PART_CODES = 0, HIFA4_PART_META = 1, HIFA4_PART_MMA = 2, HIFA4_PART_AUX = 3 }; /* `part` */
 enum { HIFA4_MAX_HEADS = 256, HIFA4_MAX_DEBUG_BLOCKS = 16 };
 #define HIFA4_STATIC_CALIB_MAX_FLOATS (1u << 20)   /* scratch limit of hifa4_smooth_calibrate_static */
 
@@ -74,11 +74,19 @@ typedef struct {
  * Groups run along each GEMM's contraction axis: along d for Q and K
  * (codes [B,H,N,d/2], meta [B,H,N,d/64], mma [B,H,N,d]); along tokens for V
  * (codes [B,Hkv,d,N/2], meta [B,Hkv,d,N/64], mma [B,Hkv,d,N], i.e. V is
- * stored transposed). */
+ * stored transposed).
+ * Q-Mean auxiliary (Algorithm 1 lines 2 and 6; "Auxiliary Q-Mean Compensation"): when q_mu and
+ * k_sum are both non-NULL, hifa4_quantize_qkv subtracts from every smoothed query token its mean
+ * over the d channels before quantizing (the Q buffers then hold Q_z) and writes
+ *   q_mu  [B,Hq,N]  floats: the per-token mean mu_i, an FP16 value;
+ *   k_sum [B,Hkv,N] floats: sum over channels of the smoothed key, an FP16 value;
+ * hifa4_attention_fwd with prm->qmean = 1 adds mu_i * k_sum_j to the raw score accumulators.
+ * Leave both NULL for the path without Q-Mean.  (hifa4_quant_bytes: part HIFA4_PART_AUX.) */
 typedef struct {
     uint8_t* q_codes; uint32_t* q_meta; void* q_mma;
     uint8_t* k_codes; uint32_t* k_meta; void* k_mma;
     uint8_t* v_codes; uint32_t* v_meta; void* v_mma;
+    float* q_mu; float* k_sum;
 } hifa4_qkv;
 
 /* Calibration result summary (host memory).  rho_K and T_KQ are the gate
@@ -94,7 +102,9 @@ typedef struct { float rho_K, T_KQ; int branch; float alpha; } hifa4_calib_stats
  *               holds after each Bc keys (Algorithm 1 lines 7-10).
  *   normalizer  0: consistent (P-Reordering, normalizer = rowsum of P-hat via
  *               the ones column); 1 (mismatched) is not built.
- *   qmean       must be 0 (Q-Mean auxiliary, Algorithm 1 lines 2 and 6, not built).
+ *   qmean       1: add the Q-Mean correction mu_i * k_sum_j to the raw scores (line 6; scaled by the
+ *               softmax scale together with them); needs qkv->q_mu and qkv->k_sum filled by
+ *               hifa4_quantize_qkv.  0: no correction (the Q buffers must then hold un-centred Q).
  *   p_dtype     HIFA4_F16: exp(S-m) is rounded to FP16 before quantization
  *               ("FP16 operations", Appendix "Implementation Details").
  *   out_dtype   HIFA4_F16 / HIFA4_BF16 / HIFA4_F32 element type of `out`.
@@ -196,8 +206,9 @@ int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv,
                         const hifa4_attn_params* prm, void* out, void* workspace,
                         const hifa4_debug* dbg, int* d_status, void* stream);
 
-/* Workspace for hifa4_attention_fwd_raw: all nine hifa4_qkv buffers (each
- * rounded up to 256 bytes) plus the attention workspace. */
+/* Workspace for hifa4_attention_fwd_raw: all hifa4_qkv buffers (each rounded up
+ * to 256 bytes; the two Q-Mean vectors only when prm->qmean = 1) plus the
+ * attention workspace. */
 size_t hifa4_attention_raw_workspace_bytes(const hifa4_shape* shape, const hifa4_attn_params* prm);
 
 /* Algorithm 1 end to end on raw post-RoPE Q/K/V: hifa4_quantize_qkv into

@@ -268,6 +268,48 @@ int hifa4_oracle_smooth_calibrate(const float* q_cal, const float* k_cal, int S,
 }
 
 /* ------------------------------------------------------------------ */
+/* Q-Mean auxiliary (Algorithm 1 lines 2 and 6; Appendix, "Q-Mean GEMV  */
+/* and coordinate consistency").                                       */
+/* ------------------------------------------------------------------ */
+
+/* Line 2 on one smoothed query row qt[d] (in place): mu = mean over the d channels, kept in FP16
+ * (exact = 1 keeps it in double); q_z = qt - mu rounded to the activation dtype (3 = no rounding). */
+double hifa4_oracle_qmean_row(double* qt, int d, int dtype, int exact)
+{
+    double mu = 0;
+    for (int c = 0; c < d; ++c) mu += qt[c];
+    mu /= d;
+    if (!exact) mu = hifa4_oracle_rn_f16(mu);
+    for (int c = 0; c < d; ++c) qt[c] = dtype == 3 ? qt[c] - mu : round_dtype(qt[c] - mu, dtype);
+    return mu;
+}
+
+/* The key-side vector of line 6: sum over channels of the smoothed key, kept in FP16. */
+double hifa4_oracle_ksum_row(const double* kt, int d, int exact)
+{
+    double a = 0;
+    for (int c = 0; c < d; ++c) a += kt[c];
+    return exact ? a : hifa4_oracle_rn_f16(a);
+}
+
+/* Bulk forms for the parity tests: x [rows][d] raw activations, scale [d] or NULL.
+ * qmean_rows: y = q_z (double), mu [rows].  ksum_rows: ks [rows]. */
+void hifa4_oracle_qmean_rows(const float* x, long rows, int d, const float* scale, int dtype,
+                             double* y, double* mu)
+{
+    hifa4_oracle_smooth_apply(x, rows, d, scale, dtype, y);
+    for (long r = 0; r < rows; ++r) mu[r] = hifa4_oracle_qmean_row(y + r * d, d, dtype, 0);
+}
+
+void hifa4_oracle_ksum_rows(const float* x, long rows, int d, const float* scale, int dtype, double* ks)
+{
+    double* y = (double*)malloc(sizeof(double) * rows * d);
+    hifa4_oracle_smooth_apply(x, rows, d, scale, dtype, y);
+    for (long r = 0; r < rows; ++r) ks[r] = hifa4_oracle_ksum_row(y + r * d, d, 0);
+    free(y);
+}
+
+/* ------------------------------------------------------------------ */
 /* Algorithm 1 for a set of query rows that share one KV head.         */
 /* ------------------------------------------------------------------ */
 
@@ -316,11 +358,7 @@ int hifa4_oracle_attention_rows(const hifa4_oracle_params* p, const float* q_row
     if (p->quant_k) hifa4_oracle_hif4_quantize_rows(kt, N, d, NULL, NULL, kh);
     else memcpy(kh, kt, sizeof(double) * N * d);
     if (p->qmean)
-        for (int j = 0; j < N; ++j) {
-            double a = 0;
-            for (int c = 0; c < d; ++c) a += kt[(long)j * d + c];
-            ksum[j] = p->state ? a : hifa4_oracle_rn_f16(a);
-        }
+        for (int j = 0; j < N; ++j) ksum[j] = hifa4_oracle_ksum_row(kt + (long)j * d, d, p->state);
     for (long i = 0; i < (long)N * d; ++i) vh[i] = v[i];
     if (p->quant_v) {
         if (p->v_axis == 1) {
@@ -353,13 +391,7 @@ int hifa4_oracle_attention_rows(const hifa4_oracle_params* p, const float* q_row
 
         hifa4_oracle_smooth_apply(q_rows + (long)row * d, 1, d, s, p->in_dtype, qt);
         double mu = 0;
-        if (p->qmean) {
-            for (int c = 0; c < d; ++c) mu += qt[c];
-            mu /= d;
-            if (!p->state) mu = hifa4_oracle_rn_f16(mu);
-            for (int c = 0; c < d; ++c)
-                qt[c] = p->in_dtype == 3 ? qt[c] - mu : round_dtype(qt[c] - mu, p->in_dtype);
-        }
+        if (p->qmean) mu = hifa4_oracle_qmean_row(qt, d, p->in_dtype, p->state);
         if (p->quant_q) hifa4_oracle_hif4_quantize_rows(qt, 1, d, NULL, NULL, qh);
         else memcpy(qh, qt, sizeof(double) * d);
 

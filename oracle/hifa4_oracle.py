@@ -134,6 +134,32 @@ def smooth_quantize(x: np.ndarray, scale, dtype: int, axis_tokens: bool = False)
     return hif4_quantize_rows(y)
 
 
+def qmean_quantize(x: np.ndarray, scale, dtype: int):
+    """Algorithm 1 lines 1-3 for Q with the Q-Mean auxiliary: smooth, subtract the per-token mean
+    (kept in FP16), round to the activation dtype, HIF4 along channels.
+    x [..., N, d]; returns (codes, meta, deq, mu [..., N])."""
+    x = np.ascontiguousarray(x, np.float32)
+    d = x.shape[-1]
+    rows = x.size // d
+    y = np.empty(x.shape, np.float64)
+    mu = np.empty(x.shape[:-1], np.float64)
+    sc = None if scale is None else np.ascontiguousarray(scale, np.float32)
+    lib().hifa4_oracle_qmean_rows(_p(x, C.c_float), C.c_long(rows), C.c_int(d), _p(sc, C.c_float),
+                                  C.c_int(dtype), _p(y, C.c_double), _p(mu, C.c_double))
+    return hif4_quantize_rows(y) + (mu,)
+
+
+def ksum_rows(x: np.ndarray, scale, dtype: int) -> np.ndarray:
+    """Sum over channels of the smoothed key, kept in FP16 (Algorithm 1 line 6).  x [..., N, d]."""
+    x = np.ascontiguousarray(x, np.float32)
+    d = x.shape[-1]
+    ks = np.empty(x.shape[:-1], np.float64)
+    sc = None if scale is None else np.ascontiguousarray(scale, np.float32)
+    lib().hifa4_oracle_ksum_rows(_p(x, C.c_float), C.c_long(x.size // d), C.c_int(d), _p(sc, C.c_float),
+                                 C.c_int(dtype), _p(ks, C.c_double))
+    return ks
+
+
 def smooth_calibrate(q_cal: np.ndarray, k_cal: np.ndarray, mode: int, alpha: float = 0.0,
                      q_to_kv=None):
     """q_cal [S,Hq,Ncal,d], k_cal [S,Hkv,Ncal,d] -> dict(s, inv_s, kagg, qagg, stats)."""

@@ -15,7 +15,7 @@ from . import build as _build
 
 F16, BF16, F32 = 0, 1, 2
 Q, K, V = 0, 1, 2
-CODES, META, MMA = 0, 1, 2
+CODES, META, MMA, AUX = 0, 1, 2, 3
 MODE_BYPASS, MODE_STRONG, MODE_MILD, MODE_AUTO, MODE_CUSTOM = 0, 1, 2, 3, 4
 MAX_DEBUG_BLOCKS = 16
 
@@ -36,7 +36,7 @@ class _Shape(C.Structure):
 
 class _QKV(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("q_codes", "q_meta", "q_mma", "k_codes", "k_meta", "k_mma",
-                                          "v_codes", "v_meta", "v_mma")]
+                                          "v_codes", "v_meta", "v_mma", "q_mu", "k_sum")]
 
 
 class _AttnParams(C.Structure):
@@ -171,10 +171,14 @@ class QuantizedQKV:
     v_codes: torch.Tensor
     v_meta: torch.Tensor
     v_mma: torch.Tensor
+    q_mu: torch.Tensor | None = None        # Q-Mean auxiliary: per-token mean of the smoothed query
+    k_sum: torch.Tensor | None = None       # Q-Mean auxiliary: channel sum of the smoothed key
 
     def struct(self) -> _QKV:
-        return _QKV(*[getattr(self, n).data_ptr() for n in ("q_codes", "q_meta", "q_mma", "k_codes",
-                                                            "k_meta", "k_mma", "v_codes", "v_meta", "v_mma")])
+        ptrs = [getattr(self, n).data_ptr() for n in ("q_codes", "q_meta", "q_mma", "k_codes",
+                                                      "k_meta", "k_mma", "v_codes", "v_meta", "v_mma")]
+        ptrs += [None if t is None else t.data_ptr() for t in (self.q_mu, self.k_sum)]
+        return _QKV(*ptrs)
 
 
 def quant_bytes(B, Hq, Hkv, N, d, in_dtype, which, part) -> int:
@@ -182,8 +186,8 @@ def quant_bytes(B, Hq, Hkv, N, d, in_dtype, which, part) -> int:
     return int(lib().hifa4_quant_bytes(C.byref(s), which, part))
 
 
-def alloc_qkv(B, Hq, Hkv, N, d, in_dtype, device, q_to_kv=None) -> QuantizedQKV:
-    """Allocate the nine buffers with the sizes the library reports."""
+def alloc_qkv(B, Hq, Hkv, N, d, in_dtype, device, q_to_kv=None, qmean=False) -> QuantizedQKV:
+    """Allocate the buffers with the sizes the library reports (qmean: also the two Q-Mean vectors)."""
     bufs = {}
     for w, name, H in ((Q, "q", Hq), (K, "k", Hkv), (V, "v", Hkv)):
         nb = [quant_bytes(B, Hq, Hkv, N, d, in_dtype, w, p) for p in (CODES, META, MMA)]
@@ -197,6 +201,10 @@ def alloc_qkv(B, Hq, Hkv, N, d, in_dtype, device, q_to_kv=None) -> QuantizedQKV:
         bufs[name + "_mma"] = torch.empty(lead + (ln,), dtype=torch.bfloat16, device=device)
         assert bufs[name + "_codes"].numel() == nb[0] and bufs[name + "_meta"].numel() * 4 == nb[1]
         assert bufs[name + "_mma"].numel() * 2 == nb[2]
+    if qmean:
+        assert quant_bytes(B, Hq, Hkv, N, d, in_dtype, Q, AUX) == B * Hq * N * 4
+        bufs["q_mu"] = torch.empty((B, Hq, N), dtype=torch.float32, device=device)
+        bufs["k_sum"] = torch.empty((B, Hkv, N), dtype=torch.float32, device=device)
     return QuantizedQKV(B, Hq, Hkv, N, d, in_dtype, q_to_kv, **bufs)
 
 
@@ -240,14 +248,15 @@ def smooth_calibrate_static(q_cal, k_cal, mode, alpha=0.0, q_to_kv=None, s=None,
 
 
 def quantize_qkv(q, k, v, s=None, inv_s=None, q_to_kv=None, out: QuantizedQKV | None = None,
-                 d_status=None) -> QuantizedQKV:
-    """Smooth-QK + HIF4 quantization of device tensors q [B,Hq,N,d], k, v [B,Hkv,N,d]."""
+                 d_status=None, qmean=False) -> QuantizedQKV:
+    """Smooth-QK + HIF4 quantization of device tensors q [B,Hq,N,d], k, v [B,Hkv,N,d].
+    qmean: also apply the Q-Mean auxiliary (the Q buffers then hold the mean-free Q_z)."""
     assert q.is_cuda and q.is_contiguous() and k.is_contiguous() and v.is_contiguous()
     B, Hq, N, d = q.shape
     Hkv = k.shape[1]
     dt = _DT[q.dtype]
     if out is None:
-        out = alloc_qkv(B, Hq, Hkv, N, d, dt, q.device, q_to_kv)
+        out = alloc_qkv(B, Hq, Hkv, N, d, dt, q.device, q_to_kv, qmean=qmean)
     sh = _shape(B, Hq, Hkv, N, d, dt, q_to_kv)
     st = out.struct()
     rc = lib().hifa4_quantize_qkv(C.byref(sh), _ptr(q), _ptr(k), _ptr(v), _ptr(s), _ptr(inv_s),
@@ -257,12 +266,12 @@ def quantize_qkv(q, k, v, s=None, inv_s=None, q_to_kv=None, out: QuantizedQKV | 
 
 
 def attention_fwd(qkv: QuantizedQKV, causal: bool, Bc: int = 128, out_dtype=F32, out=None,
-                  debug_blocks=None, d_status=None, softmax_scale=0.0, Br=128):
+                  debug_blocks=None, d_status=None, softmax_scale=0.0, Br=128, qmean=False):
     """Fused attention forward on quantized operands.  Returns out [B,Hq,N,d], or
     (out, dict(p_codes, p_step, l, m)) when debug_blocks (a list of (b, h, query block)) is given."""
     dev = qkv.q_mma.device
     sh = _shape(qkv.B, qkv.Hq, qkv.Hkv, qkv.N, qkv.d, qkv.in_dtype, qkv.q_to_kv)
-    prm = _params(causal, Bc, out_dtype, Br=Br, softmax_scale=softmax_scale)
+    prm = _params(causal, Bc, out_dtype, Br=Br, softmax_scale=softmax_scale, qmean=int(qmean))
     if out is None:
         out = torch.empty((qkv.B, qkv.Hq, qkv.N, qkv.d), dtype=_TORCH_DT[out_dtype], device=dev)
     st = qkv.struct()
@@ -285,20 +294,20 @@ def attention_fwd(qkv: QuantizedQKV, causal: bool, Bc: int = 128, out_dtype=F32,
     return (out, dump) if debug_blocks else out
 
 
-def attention_raw_workspace_bytes(B, Hq, Hkv, N, d, in_dtype, causal, Bc, out_dtype=F32) -> int:
+def attention_raw_workspace_bytes(B, Hq, Hkv, N, d, in_dtype, causal, Bc, out_dtype=F32, qmean=False) -> int:
     sh = _shape(B, Hq, Hkv, N, d, in_dtype)
-    prm = _params(causal, Bc, out_dtype)
+    prm = _params(causal, Bc, out_dtype, qmean=int(qmean))
     return int(lib().hifa4_attention_raw_workspace_bytes(C.byref(sh), C.byref(prm)))
 
 
 def attention_fwd_raw(q, k, v, s, inv_s, causal: bool, Bc: int = 128, out_dtype=F32, q_to_kv=None,
-                      out=None, workspace=None, d_status=None, softmax_scale=0.0):
+                      out=None, workspace=None, d_status=None, softmax_scale=0.0, qmean=False):
     """Algorithm 1 end to end on raw device tensors (quantize into the workspace, then attend)."""
     B, Hq, N, d = q.shape
     Hkv = k.shape[1]
     dt = _DT[q.dtype]
     sh = _shape(B, Hq, Hkv, N, d, dt, q_to_kv)
-    prm = _params(causal, Bc, out_dtype, softmax_scale=softmax_scale)
+    prm = _params(causal, Bc, out_dtype, softmax_scale=softmax_scale, qmean=int(qmean))
     need = int(lib().hifa4_attention_raw_workspace_bytes(C.byref(sh), C.byref(prm)))
     if need == 0:
         raise Hifa4Error(2, "hifa4_attention_raw_workspace_bytes")

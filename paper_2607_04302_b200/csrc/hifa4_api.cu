@@ -116,10 +116,11 @@ int hifa4_smooth_calibrate(const void* q_cal, const void* k_cal, int S, int Hq, 
 size_t hifa4_quant_bytes(const hifa4_shape* shape, int which, int part)
 {
     if (check_shape(shape) != HIFA4_OK) return 0;
-    if (which < HIFA4_Q || which > HIFA4_V || part < HIFA4_PART_CODES || part > HIFA4_PART_MMA) return 0;
+    if (which < HIFA4_Q || which > HIFA4_V || part < HIFA4_PART_CODES || part > HIFA4_PART_AUX) return 0;
     size_t H = which == HIFA4_Q ? shape->Hq : shape->Hkv;
     size_t elems = (size_t)shape->B * H * shape->N * shape->d;
     switch (part) {
+    case HIFA4_PART_AUX: return which == HIFA4_V ? 0 : elems / shape->d * sizeof(float);
     case HIFA4_PART_CODES: return elems / 2;
     case HIFA4_PART_META: return elems / 64 * 4;
     default: return elems * 2;
@@ -138,15 +139,16 @@ int hifa4_quantize_qkv(const hifa4_shape* shape, const void* q, const void* k, c
     if (q && (!out->q_codes || !out->q_meta || !out->q_mma)) return HIFA4_ERR_INVALID_ARG;
     if (k && (!out->k_codes || !out->k_meta || !out->k_mma)) return HIFA4_ERR_INVALID_ARG;
     if (v && (!out->v_codes || !out->v_meta || !out->v_mma)) return HIFA4_ERR_INVALID_ARG;
+    if ((out->q_mu == nullptr) != (out->k_sum == nullptr)) return HIFA4_ERR_INVALID_ARG;
     HeadMap qmap, kmap;
     if ((rc = build_map(shape->Hq, shape->Hkv, shape->q_to_kv, qmap, kmap))) return rc;
     if ((rc = check_arch())) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     const int B = shape->B, N = shape->N, d = shape->d, dt = shape->in_dtype;
     if (q && launch_quantize_rows(dt, q, s, qmap, B, shape->Hq, N, d, out->q_codes, out->q_meta,
-                                  out->q_mma, st) != cudaSuccess) return HIFA4_ERR_CUDA;
+                                  out->q_mma, out->q_mu, nullptr, st) != cudaSuccess) return HIFA4_ERR_CUDA;
     if (k && launch_quantize_rows(dt, k, inv_s, kmap, B, shape->Hkv, N, d, out->k_codes, out->k_meta,
-                                  out->k_mma, st) != cudaSuccess) return HIFA4_ERR_CUDA;
+                                  out->k_mma, nullptr, out->k_sum, st) != cudaSuccess) return HIFA4_ERR_CUDA;
     if (v && launch_quantize_tokens(dt, v, B, shape->Hkv, N, d, out->v_codes, out->v_meta,
                                     out->v_mma, st) != cudaSuccess) return HIFA4_ERR_CUDA;
     return HIFA4_OK;
@@ -162,7 +164,8 @@ static int check_attn(const hifa4_shape* shape, const hifa4_attn_params* prm)
     if (prm->Br != 128) return HIFA4_ERR_UNSUPPORTED;
     if (prm->Bc != 64 && prm->Bc != 128) return HIFA4_ERR_UNSUPPORTED;
     if (shape->d == 256 && prm->Bc != 64) return HIFA4_ERR_UNSUPPORTED;
-    if (prm->normalizer != 0 || prm->qmean != 0 || prm->p_dtype != HIFA4_F16) return HIFA4_ERR_UNSUPPORTED;
+    if (prm->qmean != 0 && prm->qmean != 1) return HIFA4_ERR_INVALID_ARG;
+    if (prm->normalizer != 0 || prm->p_dtype != HIFA4_F16) return HIFA4_ERR_UNSUPPORTED;
     return HIFA4_OK;
 }
 
@@ -181,6 +184,7 @@ int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv, const hi
     int rc = check_attn(shape, prm);
     if (rc) return rc;
     if (!qkv || !out || !qkv->q_mma || !qkv->k_mma || !qkv->v_mma) return HIFA4_ERR_INVALID_ARG;
+    if (prm->qmean && (!qkv->q_mu || !qkv->k_sum)) return HIFA4_ERR_INVALID_ARG;
     if (dbg) {
         if (dbg->n_blocks < 0 || dbg->n_blocks > HIFA4_MAX_DEBUG_BLOCKS) return HIFA4_ERR_INVALID_ARG;
         if (dbg->n_blocks > 0 && !dbg->blocks) return HIFA4_ERR_INVALID_ARG;
@@ -197,7 +201,7 @@ int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv, const hi
     return launch_attention(*shape, qmap, *qkv, *prm, out, dbg, d_status, (cudaStream_t)stream);
 }
 
-static size_t qkv_layout(const hifa4_shape* shape, char* base, hifa4_qkv* o)
+static size_t qkv_layout(const hifa4_shape* shape, int qmean, char* base, hifa4_qkv* o)
 {
     size_t off = 0;
     void** slots[9] = {(void**)&o->q_codes, (void**)&o->q_meta, &o->q_mma,
@@ -208,13 +212,20 @@ static size_t qkv_layout(const hifa4_shape* shape, char* base, hifa4_qkv* o)
             if (o) *slots[3 * w + p] = base + off;
             off += align256(hifa4_quant_bytes(shape, w, p));
         }
+    if (o) { o->q_mu = nullptr; o->k_sum = nullptr; }
+    if (qmean) {
+        if (o) o->q_mu = (float*)(base + off);
+        off += align256(hifa4_quant_bytes(shape, HIFA4_Q, HIFA4_PART_AUX));
+        if (o) o->k_sum = (float*)(base + off);
+        off += align256(hifa4_quant_bytes(shape, HIFA4_K, HIFA4_PART_AUX));
+    }
     return off;
 }
 
 size_t hifa4_attention_raw_workspace_bytes(const hifa4_shape* shape, const hifa4_attn_params* prm)
 {
     if (check_attn(shape, prm) != HIFA4_OK) return 0;
-    return qkv_layout(shape, nullptr, nullptr) + hifa4_attention_workspace_bytes(shape, prm);
+    return qkv_layout(shape, prm->qmean, nullptr, nullptr) + hifa4_attention_workspace_bytes(shape, prm);
 }
 
 int hifa4_attention_fwd_raw(const hifa4_shape* shape, const void* q, const void* k, const void* v,
@@ -228,7 +239,7 @@ int hifa4_attention_fwd_raw(const hifa4_shape* shape, const void* q, const void*
     size_t need = hifa4_attention_raw_workspace_bytes(shape, prm);
     if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) return HIFA4_ERR_WORKSPACE;
     hifa4_qkv bufs;
-    size_t used = qkv_layout(shape, (char*)workspace, &bufs);
+    size_t used = qkv_layout(shape, prm->qmean, (char*)workspace, &bufs);
     if ((rc = hifa4_quantize_qkv(shape, q, k, v, s, inv_s, &bufs, d_status, stream))) return rc;
     return hifa4_attention_fwd(shape, &bufs, prm, out, (char*)workspace + used, nullptr, d_status, stream);
 }

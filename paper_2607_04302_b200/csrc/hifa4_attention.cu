@@ -80,6 +80,9 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
         const int n_tiles = last_key / BC + 1;
         float m_run = -INFINITY;                          // FP16 value held in a float
         const float LOG2E = 1.4426950408889634f;
+        // Q-Mean correction (line 6): mu of this row, channel sum of every key of the KV head
+        const float mu_row = (args.qmean && row < N) ? args.q_mu[(size_t)bh_q * N + row] : 0.f;
+        auto ksum_of = [&](int key) { return key < N ? __ldg(args.k_sum + (size_t)bh_kv * N + key) : 0.f; };
         constexpr uint32_t idesc_s = umma_idesc_bf16(128, BC);
         constexpr uint32_t idesc_o = umma_idesc_bf16(128, (C::O_COLS <= 256) ? C::O_COLS : 256);
         constexpr uint32_t idesc_l = umma_idesc_bf16(128, 16);
@@ -126,6 +129,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
                     float a = __uint_as_float(r[i]);
+                    if (args.qmean) a = fmaf(mu_row, ksum_of(j0 + cc * 32 + i), a);
                     if (need_mask && (j0 + cc * 32 + i > key_lim)) a = -INFINITY;
                     mx = fmaxf(mx, a);
                 }
@@ -162,7 +166,9 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
                     tmem_wait_ld();
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        float t = fmaf(__uint_as_float(r[i]), args.c1, -mL);
+                        float a = __uint_as_float(r[i]);
+                        if (args.qmean) a = fmaf(mu_row, ksum_of(j0 + gq * 64 + cc * 32 + i), a);
+                        float t = fmaf(a, args.c1, -mL);
                         float e = f16_round(ex2_approx(t));
                         if (need_mask && (j0 + gq * 64 + cc * 32 + i > key_lim)) e = 0.f;
                         p[cc * 32 + i] = e;
@@ -327,6 +333,9 @@ int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv&
     a.c0 = (float)sigma;
     a.c1 = (float)(sigma * 1.4426950408889634074);
     a.out = out;
+    a.qmean = prm.qmean ? 1 : 0;
+    a.q_mu = qkv.q_mu;
+    a.k_sum = qkv.k_sum;
     a.d_status = d_status;
     a.map = map;
     if (dbg && dbg->n_blocks > 0) {

@@ -24,6 +24,9 @@ struct AttnArgs {
     int B, Hq, Hkv, N;
     int causal, out_dtype;
     float c0, c1;                 // sigma, sigma * log2(e)
+    int qmean;                    // add mu_i * k_sum_j to the raw scores (Algorithm 1 line 6)
+    const float* q_mu;            // [B,Hq,N]
+    const float* k_sum;           // [B,Hkv,N]
     void* out;
     int* d_status;
     HeadMap map;

@@ -101,7 +101,7 @@ struct Schedule {
     }
 };
 
-template <int KS, bool DBG>
+template <int KS, bool DBG, bool QM>
 __global__ void __launch_bounds__((4 * KS + 2) * 32, 1)
 attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                         const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnArgs args)
@@ -292,7 +292,7 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
         // current tile is still being quantized (S is double-buffered), so the row-maximum exchange of
         // a tile is usually complete by the time its turn comes and the KS warps of a row quarter need
         // not run in phase.  g: global tile index; jt, q0: the tile's place in its own item.
-        auto fetch_scores = [&](int g, int jt, int q0, float (&sc)[KPT]) -> float {
+        auto fetch_scores = [&](int g, int jt, int q0, float mu, int bh_kv, float (&sc)[KPT]) -> float {
             const int j0 = jt * BC, kb = j0 + kq * KPT;
             const int key_lim = args.causal ? min(q0 + r_loc, N - 1) : N - 1;
             const uint32_t t_src = t_lane + S_COL + (g & 1) * 128 + kq * KPT;
@@ -303,6 +303,17 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 tmem_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 32; ++i) sc[cc * 32 + i] = __uint_as_float(r[i]);
+            }
+            if (QM && kb < N) {                                // Q-Mean correction (line 6): + mu_i * sum_c k~_jc
+                const float4* kp = reinterpret_cast<const float4*>(args.k_sum + (size_t)bh_kv * N + kb);
+#pragma unroll
+                for (int i = 0; i < KPT / 4; ++i) {
+                    const float4 ks = __ldg(kp + i);
+                    sc[4 * i] = fmaf(mu, ks.x, sc[4 * i]);
+                    sc[4 * i + 1] = fmaf(mu, ks.y, sc[4 * i + 1]);
+                    sc[4 * i + 2] = fmaf(mu, ks.z, sc[4 * i + 2]);
+                    sc[4 * i + 3] = fmaf(mu, ks.w, sc[4 * i + 3]);
+                }
             }
             const bool need_mask = (args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N);
             if (need_mask) {                                   // masked scores become -inf: exp gives exact zeros
@@ -323,6 +334,9 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             return t4[0];
         };
 
+        auto mu_of = [&](const WorkItem& w) -> float {        // Q-Mean: mean of this thread's query row
+            return (QM && w.q0 + r_loc < N) ? args.q_mu[(size_t)w.bh_q * N + w.q0 + r_loc] : 0.f;
+        };
         float pn[KPT];                                        // scores of the next tile
         float mx_next = -INFINITY;
         int g = 0;                                            // global index of the current tile
@@ -332,7 +346,7 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             if (ok) {
                 if (wait_or_abort(bar(BAR_SF), 0, abort_flag)) {
                     tc_fence_after();
-                    mx_next = fetch_scores(0, 0, first.q0, pn);
+                    mx_next = fetch_scores(0, 0, first.q0, mu_of(first), first.bh_kv, pn);
                     if (first.n_tiles == 1 && n_my > 1) ok = copy_q(1);   // S of the item's last tile has been seen
                 } else { fail(8); ok = false; }
             }
@@ -350,6 +364,7 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
             float m_run = -INFINITY;
             const bool has_next = k + 1 < n_my;
             const WorkItem nxt = has_next ? sched.item(k + 1, args) : it;   // decoded once per item, not per tile
+            const float mu_cur = mu_of(it), mu_nxt = mu_of(nxt);
 
             for (int jt = 0; ok && jt < n_tiles; ++jt, ++g) {
                 const int j0 = jt * BC;
@@ -400,7 +415,8 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                         const int n_q0 = in_item ? q0 : nxt.q0, n_nt = in_item ? n_tiles : nxt.n_tiles;
                         if (!wait_or_abort(bar(BAR_SF + (sb ^ 1)), (uint32_t)((g + 1) >> 1) & 1u, abort_flag)) { fail(8); ok = false; break; }
                         tc_fence_after();
-                        mx_next = fetch_scores(g + 1, njt, n_q0, pn);
+                        mx_next = fetch_scores(g + 1, njt, n_q0, in_item ? mu_cur : mu_nxt,
+                                               in_item ? it.bh_kv : nxt.bh_kv, pn);
                         // S of the last tile of item nk has been seen, so every QK of that item is complete and
                         // the Q-hat image in tensor memory may be replaced by the next item's
                         if (njt == n_nt - 1 && nk + 1 < n_my) {
@@ -512,11 +528,11 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     if (warp == W_MMA) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
 }
 
-template <int KS, bool DBG>
+template <int KS, bool DBG, bool QM>
 static int launch_ws(const hifa4_shape& sh, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                      const AttnArgs& args, cudaStream_t st)
 {
-    auto kern = attention_fwd_ws_kernel<KS, DBG>;
+    auto kern = attention_fwd_ws_kernel<KS, DBG, QM>;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ws::SMEM_BYTES) != cudaSuccess)
@@ -543,9 +559,11 @@ int launch_attention_ws(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnA
     if (!make_bf16_map(&mq, qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, ws::D, 128)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, ws::D, ws::BC)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, ws::D, sh.N, ws::D)) return HIFA4_ERR_CUDA;
-    // the P-hat dump code lives in a separate instantiation so that the timed path carries none of it
-    if (args.dbg.n_blocks > 0) return launch_ws<4, true>(sh, mq, mk, mv, args, st);
-    return launch_ws<4, false>(sh, mq, mk, mv, args, st);
+    // the P-hat dump code and the Q-Mean correction live in separate instantiations, so that the
+    // timed path carries none of either
+    const bool dbg = args.dbg.n_blocks > 0;
+    if (args.qmean) return dbg ? launch_ws<4, true, true>(sh, mq, mk, mv, args, st) : launch_ws<4, false, true>(sh, mq, mk, mv, args, st);
+    return dbg ? launch_ws<4, true, false>(sh, mq, mk, mv, args, st) : launch_ws<4, false, false>(sh, mq, mk, mv, args, st);
 }
 
 }  // namespace hifa4

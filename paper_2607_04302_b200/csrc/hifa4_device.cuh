@@ -76,10 +76,12 @@ template <typename T> struct In16;
 template <> struct In16<__half> {
     static __device__ __forceinline__ float to_f(uint16_t u) { return __half2float(__ushort_as_half(u)); }
     static __device__ __forceinline__ float round(float x) { return __half2float(__float2half_rn(x)); }
+    static __device__ __forceinline__ float round_d(double x) { return __half2float(__double2half(x)); }
 };
 template <> struct In16<__nv_bfloat16> {
     static __device__ __forceinline__ float to_f(uint16_t u) { return __uint_as_float((uint32_t)u << 16); }
     static __device__ __forceinline__ float round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+    static __device__ __forceinline__ float round_d(double x) { return __bfloat162float(__double2bfloat16(x)); }
 };
 
 }  // namespace hifa4

@@ -10,9 +10,10 @@ struct HeadMap;
 
 void count_launch();
 
+// mu_out: subtract the per-row mean (Q-Mean) and write it; ksum_out: write the per-row channel sum.
 cudaError_t launch_quantize_rows(int dtype, const void* x, const float* scale, const HeadMap& map,
                                  int B, int H, int N, int d, uint8_t* codes, uint32_t* meta,
-                                 void* img, cudaStream_t st);
+                                 void* img, float* mu_out, float* ksum_out, cudaStream_t st);
 cudaError_t launch_quantize_tokens(int dtype, const void* x, int B, int H, int N, int d,
                                    uint8_t* codes, uint32_t* meta, void* img, cudaStream_t st);
 cudaError_t launch_absmax(int dtype, const void* x, const HeadMap& map, int S, int H, int Hkv,

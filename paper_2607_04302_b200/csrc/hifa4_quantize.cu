@@ -71,7 +71,8 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 quantize_rows_kernel(const uint16_t* __restrict__ x, const float* __restrict__ scale, HeadMap map,
                      int H, int N, int d, long long n_units, uint8_t* __restrict__ codes,
-                     uint32_t* __restrict__ meta, uint16_t* __restrict__ img)
+                     uint32_t* __restrict__ meta, uint16_t* __restrict__ img,
+                     float* __restrict__ mu_out, float* __restrict__ ksum_out)
 {
     long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= n_units) return;                        // n_units % 32 == 0: whole warps leave together
@@ -90,6 +91,23 @@ quantize_rows_kernel(const uint16_t* __restrict__ x, const float* __restrict__ s
         const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
 #pragma unroll
         for (int i = 0; i < 8; ++i) v[i] = In16<T>::round(v[i] * sv[i]);
+    }
+    if (mu_out || ksum_out) {
+        // Q-Mean auxiliary (Algorithm 1 lines 2 and 6).  A row of d channels sits in d/8 consecutive,
+        // aligned lanes; the sum runs in double, where it is exact for any row whose values span fewer
+        // than ~40 binades, so its order does not matter.
+        double sum = 0.0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sum += (double)v[i];
+        for (int off = 1; off < d / 8; off <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+        if (mu_out) {                                // q_z = round_in(q~ - mu), mu = FP16(mean)
+            const float mu = __half2float(__double2half(sum / (double)d));
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = In16<T>::round_d((double)v[i] - (double)mu);
+            if (c0 == 0) mu_out[row] = mu;
+        } else if (c0 == 0) {
+            ksum_out[row] = __half2float(__double2half(sum));
+        }
     }
     float dq[8];
     uint32_t mw;
@@ -183,23 +201,24 @@ __global__ void smooth_finalize_kernel(const float* __restrict__ kmax, const flo
 // ------------------------------------------------------------------------------- launchers
 template <typename T>
 static cudaError_t launch_rows(const void* x, const float* scale, const HeadMap& map, int B, int H,
-                               int N, int d, uint8_t* codes, uint32_t* meta, void* img,
-                               cudaStream_t st)
+                               int N, int d, uint8_t* codes, uint32_t* meta, void* img, float* mu_out,
+                               float* ksum_out, cudaStream_t st)
 {
     long long units = (long long)B * H * N * d / 8;
     unsigned blocks = (unsigned)((units + 255) / 256);
     quantize_rows_kernel<T><<<blocks, 256, 0, st>>>((const uint16_t*)x, scale, map, H, N, d, units,
-                                                    codes, meta, (uint16_t*)img);
+                                                    codes, meta, (uint16_t*)img, mu_out, ksum_out);
     count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_quantize_rows(int dtype, const void* x, const float* scale, const HeadMap& map,
                                  int B, int H, int N, int d, uint8_t* codes, uint32_t* meta,
-                                 void* img, cudaStream_t st)
+                                 void* img, float* mu_out, float* ksum_out, cudaStream_t st)
 {
-    return dtype == HIFA4_F16 ? launch_rows<__half>(x, scale, map, B, H, N, d, codes, meta, img, st)
-                              : launch_rows<__nv_bfloat16>(x, scale, map, B, H, N, d, codes, meta, img, st);
+    return dtype == HIFA4_F16
+               ? launch_rows<__half>(x, scale, map, B, H, N, d, codes, meta, img, mu_out, ksum_out, st)
+               : launch_rows<__nv_bfloat16>(x, scale, map, B, H, N, d, codes, meta, img, mu_out, ksum_out, st);
 }
 
 cudaError_t launch_quantize_tokens(int dtype, const void* x, int B, int H, int N, int d,

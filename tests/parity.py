@@ -34,8 +34,9 @@ def calibrate(cfg, device):
     return hb.smooth_calibrate(qc.to(device), kc.to(device), cfg.smooth_mode)
 
 
-def check_quantized(cfg, q, k, v, s, inv_s, qkv):
-    """Bit-exact comparison of codes, metadata and the BF16 operand image with the oracle."""
+def check_quantized(cfg, q, k, v, s, inv_s, qkv, qmean=False):
+    """Bit-exact comparison of codes, metadata and the BF16 operand image with the oracle (and of
+    the two Q-Mean vectors when qmean is set)."""
     dt = orc.F16 if cfg.dtype == "fp16" else orc.BF16
     s_np = None if s is None else np32(s)
     is_np = None if inv_s is None else np32(inv_s)
@@ -45,9 +46,19 @@ def check_quantized(cfg, q, k, v, s, inv_s, qkv):
                              ("k", k, is_np, False), ("v", v, None, True)):
         xn = np32(x)
         codes_l, meta_l, deq_l = [], [], []
+        aux_l = []
         for h in range(xn.shape[1]):
-            c, m, dq = orc.smooth_quantize(xn[:, h], None if sc is None else sc[h], dt, axis_tokens=tok)
+            if qmean and name == "q":
+                c, m, dq, mu = orc.qmean_quantize(xn[:, h], None if sc is None else sc[h], dt)
+                aux_l.append(mu)
+            else:
+                c, m, dq = orc.smooth_quantize(xn[:, h], None if sc is None else sc[h], dt, axis_tokens=tok)
+                if qmean and name == "k":
+                    aux_l.append(orc.ksum_rows(xn[:, h], None if sc is None else sc[h], dt))
             codes_l.append(c); meta_l.append(m); deq_l.append(dq)
+        if aux_l:
+            g_aux = getattr(qkv, "q_mu" if name == "q" else "k_sum").cpu().numpy().astype(np.float64)
+            assert np.array_equal(g_aux, np.stack(aux_l, 1)), f"{name} Q-Mean vector differs"
         codes, meta, deq = (np.stack(a, 1) for a in (codes_l, meta_l, deq_l))
         g_codes = getattr(qkv, name + "_codes").cpu().numpy()
         g_meta = getattr(qkv, name + "_meta").cpu().numpy().view(np.uint32)
@@ -58,7 +69,7 @@ def check_quantized(cfg, q, k, v, s, inv_s, qkv):
 
 
 def run_case(cfg, device="cuda:0", blocks=None, out_dtype=hb.F32, check_quant=True, rows_per_block=None,
-             qkv_host=None):
+             qkv_host=None, qmean=False):
     """Full path on the GPU + oracle on the requested 128-row query blocks.
 
     blocks: list of (b, h, query_block); default: every block (small cases only).
@@ -67,9 +78,9 @@ def run_case(cfg, device="cuda:0", blocks=None, out_dtype=hb.F32, check_quant=Tr
     s, inv_s = calibrate(cfg, device)
     qd, kd, vd = q.to(device), k.to(device), v.to(device)
     status = torch.zeros(1, dtype=torch.int32, device=device)
-    qkv = hb.quantize_qkv(qd, kd, vd, s, inv_s, d_status=status)
+    qkv = hb.quantize_qkv(qd, kd, vd, s, inv_s, d_status=status, qmean=qmean)
     if check_quant:
-        check_quantized(cfg, q, k, v, s, inv_s, qkv)
+        check_quantized(cfg, q, k, v, s, inv_s, qkv, qmean=qmean)
     n_qb = (cfg.N + 127) // 128
     if blocks is None:
         blocks = [(b, h, t) for b in range(cfg.B) for h in range(cfg.Hq) for t in range(n_qb)]
@@ -79,7 +90,7 @@ def run_case(cfg, device="cuda:0", blocks=None, out_dtype=hb.F32, check_quant=Tr
     for i0 in range(0, len(blocks), hb.MAX_DEBUG_BLOCKS):
         chunk = blocks[i0:i0 + hb.MAX_DEBUG_BLOCKS]
         out, dump = hb.attention_fwd(qkv, cfg.causal, Bc=cfg.Bc, out_dtype=out_dtype, debug_blocks=chunk,
-                                     d_status=status)
+                                     d_status=status, qmean=qmean)
         torch.cuda.synchronize()
         assert int(status.item()) == 0, f"device status {int(status.item())}"
         out_full = out
@@ -98,7 +109,7 @@ def run_case(cfg, device="cuda:0", blocks=None, out_dtype=hb.F32, check_quant=Tr
             o_ref, d = orc.attention_rows(qn[b, h, idx], idx, kn[b, g], vn[b, g],
                                           None if s_np is None else s_np[g], None if is_np is None else is_np[g],
                                           causal=cfg.causal, Bc=cfg.Bc, in_dtype=dt, out_dtype=out_dtype,
-                                          dumps=True)
+                                          qmean=int(qmean), dumps=True)
             loc = idx - r0
             code_ne = pc[bi, loc] != d["p_codes"]
             step_ne = np.repeat(ps[bi, loc] != d["p_step"], 4, axis=1)

@@ -49,7 +49,9 @@ def test_size_queries_and_validation_without_gpu(lib):
     sh = hb._shape(1, 4, 2, 128, 128, hb.BF16)
     prm = hb._params(True, 96, hb.F32)                                              # Bc
     assert lib.hifa4_attention_fwd(C.byref(sh), C.byref(st), C.byref(prm), one, None, None, None, None) == 2
-    prm = hb._params(True, 128, hb.F32, qmean=1)
+    prm = hb._params(True, 128, hb.F32, qmean=1)                                    # Q-Mean vectors missing
+    assert lib.hifa4_attention_fwd(C.byref(sh), C.byref(st), C.byref(prm), one, None, None, None, None) == 1
+    prm = hb._params(True, 128, hb.F32, normalizer=1)                               # mismatched normaliser: not built
     assert lib.hifa4_attention_fwd(C.byref(sh), C.byref(st), C.byref(prm), one, None, None, None, None) == 2
     # no sm_100 device here: a well-formed call is refused with ARCH or CUDA, never run on the CPU
     import torch

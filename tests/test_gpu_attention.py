@@ -152,3 +152,39 @@ def test_largest_sequence_properties(hb, causal):
     rel = (out / vhat[None, None, None, :].clamp_min(-1e30) - 1.0)
     rel = rel[..., vhat != 0]
     assert rel.abs().max().item() <= 2.0 ** -10                # only the FP16 rounding of the normalizer is left
+
+
+QMEAN = {
+    "qmean-d128-causal-gqa": synth.config("C2", N=512, Hq=4, Hkv=2, cal_samples=4, cal_tokens=128),
+    "qmean-d128-ragged-noncausal": synth.config("C2", N=320, Hq=2, Hkv=1, causal=False, cal_samples=4, cal_tokens=128),
+    "qmean-tiny-64x64-fp16": synth.config("C1"),
+    "qmean-d256-bc64": synth.config("C4", N=256, Hq=2, Hkv=1, Bc=64, cal_samples=3, cal_tokens=64),
+}
+
+
+@pytest.mark.parametrize("name", list(QMEAN))
+def test_qmean_auxiliary(hb, par, name):
+    """Algorithm 1 with lines 2 and 6 (Q-Mean): Q_z codes, mu, k_sum bit-exact; P-hat and output in the bars.
+    The inputs get a per-token offset on Q so that the mean is not negligible."""
+    cfg = QMEAN[name]
+    q, k, v = synth.make_qkv(cfg)
+    q = (q.float() + 0.75).to(q.dtype)
+    res = par.run_case(cfg, DEV, qkv_host=(q, k, v), qmean=True)
+    print(par.assert_within_bars(res, name))
+    # the correction matters on these inputs: without it the output differs
+    s, inv_s = par.calibrate(cfg, DEV)
+    a = hb.attention_fwd(hb.quantize_qkv(q.to(DEV), k.to(DEV), v.to(DEV), s, inv_s, qmean=True), cfg.causal, Bc=cfg.Bc, qmean=True)
+    b = hb.attention_fwd(hb.quantize_qkv(q.to(DEV), k.to(DEV), v.to(DEV), s, inv_s), cfg.causal, Bc=cfg.Bc)
+    assert not torch.equal(a, b)
+    c = hb.attention_fwd_raw(q.to(DEV), k.to(DEV), v.to(DEV), s, inv_s, cfg.causal, Bc=cfg.Bc, qmean=True)
+    assert torch.equal(a, c)
+
+
+def test_qmean_full_size_sampled(hb, par):
+    """Configuration 5 with every HiFA4 component on (Smooth-QK, Q-Mean, P-Reordering), N = 4096, B = 4."""
+    cfg = synth.config("C5", N=4096, cal_samples=2, cal_tokens=256)
+    q, k, v = synth.make_qkv(cfg)
+    q = (q.float() + 0.5).to(q.dtype)
+    blocks = [(0, 0, 0), (3, 31, 31), (1, 12, 17)]
+    res = par.run_case(cfg, DEV, blocks=blocks, check_quant=False, rows_per_block=16, qkv_host=(q, k, v), qmean=True)
+    print(par.assert_within_bars(res, "C5 N=4096 qmean"))
