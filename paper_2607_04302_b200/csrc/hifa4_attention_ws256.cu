@@ -1,0 +1,414 @@
+// Warp-specialised HiFA4 attention forward for d = 256, Bc = 64 (Algorithm 1 lines 4-13).
+//
+// One CTA = 128 query rows of one (batch, query head), 10 warps:
+//   warps 0-7  softmax / quantize: warp w owns rows 32*(w%4).. of the tile and keys 32*(w/4).. of
+//              every 64-key tile, i.e. half of the tile's single HIF4 group per thread; the two
+//              threads of a row exchange their partial score maxima through shared memory
+//   warp 8     TMA producer: Q once, then K and V^T tiles through two-stage rings
+//   warp 9     tcgen05 issuer
+// Tensor memory (512 columns): [O | l] in 0..271 (256 channels by one N = 256 MMA, the ones block by
+// an N = 16 MMA on the same A operand), the Q-hat image in 272..399, one S buffer of 64 columns at
+// 400 and the BF16 image of P-hat in 464..495.  With d = 256 there is no room for a second S buffer,
+// so S is released early instead: the softmax warps pull S(j) into registers and signal it free, and
+// S(j+1) = Q K^T runs on the tensor pipe while they work on tile j; P-hat lives in its own columns.
+// Both GEMMs take their A operand from tensor memory and only K, V^T (with its rows of ones) from
+// shared memory.  Every wait is bounded (see hifa4_attention_ws.cu for the failure protocol).
+#include "hifa4_attention.cuh"
+
+namespace hifa4 {
+
+namespace ws256 {
+constexpr int D = 256, BC = 64, STAGES = 2, KS = 2;
+constexpr int NSW = 4 * KS, THREADS = (NSW + 2) * 32, W_TMA = NSW, W_MMA = NSW + 1;
+constexpr int KPT = BC / KS, NU = KPT / 8;          // 32 keys = 4 level-2 units per thread and tile
+constexpr int Q_BYTES = 4 * 16384;                  // four 64-channel sub-tiles of 128 rows
+constexpr int K_SUB = BC * 128;                     // 64 keys x 64 channels
+constexpr int K_STAGE = 4 * K_SUB;
+constexpr int V_STAGE = (D + 16) * 128;             // 256 rows of V^T + 16 rows of ones, 64 keys wide
+constexpr int Q_OFF = 0;
+constexpr int K_OFF = Q_OFF + Q_BYTES;
+constexpr int V_OFF = K_OFF + STAGES * K_STAGE;
+constexpr int MISC_OFF = V_OFF + STAGES * V_STAGE;
+constexpr int XCHG_OFF = MISC_OFF + 256;            // partial row maxima [2 parities][2 splits][128 rows]
+constexpr int SMEM_BYTES = XCHG_OFF + 2 * 2 * 128 * 4 + 1024;
+constexpr int O_COLS = D + 16, QT_COL = 272, S_COL = 400, P_COL = 464, TMEM_COLS = 512;
+enum { BAR_Q = 0, BAR_KF = 1, BAR_KE = 3, BAR_VF = 5, BAR_VE = 7, BAR_SF = 9, BAR_SFREE = 10, BAR_PF = 11,
+       BAR_PV = 12, BAR_X = 13, BAR_QT = 17, N_BARS = 18 };
+constexpr uint32_t WAIT_POLLS = 1u << 20;
+}  // namespace ws256
+
+static __device__ __forceinline__ bool wait256(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    for (uint32_t i = 0; i < ws256::WAIT_POLLS / 64; ++i) {
+#pragma unroll 1
+        for (int j = 0; j < 64; ++j)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+    }
+    return false;
+}
+
+template <bool DBG>
+__global__ void __launch_bounds__(ws256::THREADS, 1)
+attention_fwd_ws256_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                           const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnArgs args)
+{
+    using namespace ws256;
+    if (args.d_status && *reinterpret_cast<volatile int*>(args.d_status) != 0) return;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t q_s = smem_base + Q_OFF, k_s = smem_base + K_OFF, v_s = smem_base + V_OFF,
+                   bars = smem_base + MISC_OFF;
+    auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + MISC_OFF + 8 * N_BARS);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + MISC_OFF + 8 * N_BARS + 8);
+    float* xmax = reinterpret_cast<float*>(smem_gen + XCHG_OFF);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int N = args.N;
+    const int n_qt = (N + 127) / 128;
+    // 1-D grid, query block outermost and descending: the heaviest causal CTAs are scheduled first
+    const int n_bh = args.B * args.Hq;
+    const int qt = n_qt - 1 - (int)(blockIdx.x / n_bh);
+    const int bh = (int)(blockIdx.x % n_bh);
+    const int h = bh % args.Hq, b = bh / args.Hq;
+    const int g = args.map.kv_of[h];
+    const int q0 = qt * 128;
+    const int bh_q = b * args.Hq + h, bh_kv = b * args.Hkv + g;
+    const int last_key = args.causal ? min(q0 + 127, N - 1) : N - 1;
+    const int n_tiles = last_key / BC + 1;
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(bar(BAR_Q), 1);
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar(BAR_KF + s), 1); mbar_init(bar(BAR_KE + s), 1);
+            mbar_init(bar(BAR_VF + s), 1); mbar_init(bar(BAR_VE + s), 1);
+        }
+        mbar_init(bar(BAR_SF), 1); mbar_init(bar(BAR_SFREE), NSW);
+        mbar_init(bar(BAR_PF), NSW); mbar_init(bar(BAR_PV), 1); mbar_init(bar(BAR_QT), NSW);
+        for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_X + i), KS);
+        fence_barrier_init();
+    }
+    if (warp == W_MMA) { tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS); tmem_relinquish(); }
+    if (warp == W_TMA && lane == 0) { tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_k); tma_prefetch_desc(&tmap_v); }
+    for (int i = tid; i < STAGES * 128; i += THREADS) {           // ones rows under every V^T stage
+        const int st = i / 128, off = (i % 128) * 16;
+        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};"
+                     ::"r"(v_s + st * V_STAGE + D * 128 + off), "r"(0x3F803F80u) : "memory");
+    }
+    fence_proxy_async_smem();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    auto fail = [&](int site) {
+        *abort_flag = 1;
+        if (args.d_status) atomicCAS(args.d_status, 0, HIFA4_ERR_TIMEOUT + 16 * site);
+    };
+
+    if (warp == W_TMA) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            mbar_expect_tx(bar(BAR_Q), Q_BYTES);
+#pragma unroll
+            for (int s = 0; s < 4; ++s) tma_load_3d(q_s + s * 16384, &tmap_q, bar(BAR_Q), 64 * s, q0, bh_q);
+            for (int jt = 0; jt < n_tiles; ++jt) {
+                const int st = jt & 1;
+                const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
+                const int j0 = jt * BC;
+                if (!wait256(bar(BAR_KE + st), ph ^ 1u, abort_flag)) { fail(1); break; }
+                mbar_expect_tx(bar(BAR_KF + st), K_STAGE);
+#pragma unroll
+                for (int s = 0; s < 4; ++s)
+                    tma_load_3d(k_s + st * K_STAGE + s * K_SUB, &tmap_k, bar(BAR_KF + st), 64 * s, j0, bh_kv);
+                if (!wait256(bar(BAR_VE + st), ph ^ 1u, abort_flag)) { fail(2); break; }
+                mbar_expect_tx(bar(BAR_VF + st), D * 128);
+                tma_load_3d(v_s + st * V_STAGE, &tmap_v, bar(BAR_VF + st), j0, 0, bh_kv);
+            }
+        }
+    } else if (warp == W_MMA) {
+        // ------------------------------------------------------------------ tcgen05 issuer
+        constexpr uint32_t idesc_s = umma_idesc_bf16(128, BC);
+        constexpr uint32_t idesc_o = umma_idesc_bf16(128, 256);
+        constexpr uint32_t idesc_l = umma_idesc_bf16(128, 16);
+        const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
+        const uint32_t k_lo = umma_desc_lo(k_s), v_lo = umma_desc_lo(v_s);
+        const bool leader = elect_one();
+        bool ok = true;
+        auto issue_qk = [&](int jt) {                     // S(jt) from K stage jt % 2 (16 steps of 16 channels)
+            const uint32_t b0 = k_lo + (jt & 1) * (K_STAGE >> 4);
+            if (leader) {
+#pragma unroll
+                for (int kk = 0; kk < 16; ++kk)
+                    umma_bf16_ts_lo(tm + S_COL, tm + QT_COL + kk * 8, b0 + (kk >> 2) * (K_SUB >> 4) + (kk & 3) * 2,
+                                    idesc_s, kk ? 1u : 0u);
+                umma_commit(bar(BAR_SF));
+                umma_commit(bar(BAR_KE + (jt & 1)));
+            }
+            __syncwarp();
+        };
+        ok = wait256(bar(BAR_QT), 0, abort_flag) && wait256(bar(BAR_KF), 0, abort_flag);
+        if (ok) { tc_fence_after(); issue_qk(0); } else if (leader) fail(3);
+        for (int jt = 0; ok && jt < n_tiles; ++jt) {
+            const int st = jt & 1;
+            const uint32_t ph = (uint32_t)(jt >> 1) & 1u, par = (uint32_t)jt & 1u;
+            if (jt + 1 < n_tiles) {                       // S(jt+1) as soon as S(jt) sits in registers
+                if (!wait256(bar(BAR_KF + (st ^ 1)), (uint32_t)((jt + 1) >> 1) & 1u, abort_flag)) { if (leader) fail(4); break; }
+                if (!wait256(bar(BAR_SFREE), par, abort_flag)) { if (leader) fail(5); break; }
+                tc_fence_after();
+                issue_qk(jt + 1);
+            }
+            if (!wait256(bar(BAR_VF + st), ph, abort_flag)) { if (leader) fail(6); break; }
+            if (!wait256(bar(BAR_PF), par, abort_flag)) { if (leader) fail(7); break; }
+            tc_fence_after();
+            const uint32_t b0 = v_lo + st * (V_STAGE >> 4);
+            const uint32_t acc0 = jt > 0 ? 1u : 0u;
+            if (leader) {
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {            // 16 keys per step; channels, then the ones block
+                    umma_bf16_ts_lo(tm, tm + P_COL + kk * 8, b0 + kk * 2, idesc_o, kk ? 1u : acc0);
+                    umma_bf16_ts_lo(tm + 256, tm + P_COL + kk * 8, b0 + ((D * 128) >> 4) + kk * 2, idesc_l, kk ? 1u : acc0);
+                }
+                umma_commit(bar(BAR_PV));
+                umma_commit(bar(BAR_VE + st));
+            }
+            __syncwarp();
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax / quantize
+        const int kq = warp >> 2, quarter = warp & 3;             // key half, row quarter
+        const int r_loc = quarter * 32 + lane;                    // row inside the tile = TMEM lane
+        const int row = q0 + r_loc;
+        const uint32_t t_lane = tmem + ((uint32_t)(quarter * 32) << 16);
+        const uint32_t xbar = bar(BAR_X + quarter);
+        const float LOG2E = 1.4426950408889634f;
+        const int key_lim = args.causal ? min(row, N - 1) : N - 1;
+        int dbg_slot = -1;
+        if (DBG)
+            for (int i = 0; i < args.dbg.n_blocks; ++i)
+                if (args.dbg.blocks[3 * i] == b && args.dbg.blocks[3 * i + 1] == h && args.dbg.blocks[3 * i + 2] == qt)
+                    dbg_slot = i;
+        const float mu_row = (args.qmean && row < N) ? args.q_mu[(size_t)bh_q * N + row] : 0.f;
+        float m_run = -INFINITY;
+        bool ok = true;
+
+        // Q-hat image: shared memory (swizzled TMA tiles) -> tensor memory; this thread moves 128
+        // channels of its row = 64 columns of packed BF16 pairs.
+        if (wait256(bar(BAR_Q), 0, abort_flag)) {
+            const int sw = r_loc & 7;
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t qw[32];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const int chunk = kq * 16 + half * 8 + c;          // 16-byte chunk of the 512-byte row
+                    const uint32_t a = q_s + (chunk >> 3) * 16384 + (r_loc >> 3) * 1024 + sw * 128 + (((chunk & 7) ^ sw) << 4);
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(qw[4 * c]), "=r"(qw[4 * c + 1]), "=r"(qw[4 * c + 2]), "=r"(qw[4 * c + 3]) : "r"(a));
+                }
+                tmem_st32(t_lane + QT_COL + kq * 64 + half * 32, qw);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_QT));
+        } else { fail(13); ok = false; }
+
+        for (int jt = 0; ok && jt < n_tiles; ++jt) {
+            const int j0 = jt * BC;
+            const uint32_t par = (uint32_t)jt & 1u;
+            const int kbase = j0 + kq * KPT;
+            if (!wait256(bar(BAR_SF), par, abort_flag)) { fail(8); ok = false; break; }
+            tc_fence_after();
+            float p[KPT];
+            {
+                uint32_t r[32];
+                tmem_ld32(t_lane + S_COL + kq * KPT, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) p[i] = __uint_as_float(r[i]);
+            }
+            tc_fence_before();                                 // S(jt) is in registers: S(jt+1) may overwrite it
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_SFREE));
+
+            if (args.qmean && kbase < N) {                     // Q-Mean correction (line 6): + mu_i * sum_c k~_jc
+                const float4* kp = reinterpret_cast<const float4*>(args.k_sum + (size_t)bh_kv * N + kbase);
+#pragma unroll
+                for (int i = 0; i < KPT / 4; ++i) {
+                    const float4 ks = __ldg(kp + i);
+                    p[4 * i] = fmaf(mu_row, ks.x, p[4 * i]);
+                    p[4 * i + 1] = fmaf(mu_row, ks.y, p[4 * i + 1]);
+                    p[4 * i + 2] = fmaf(mu_row, ks.z, p[4 * i + 2]);
+                    p[4 * i + 3] = fmaf(mu_row, ks.w, p[4 * i + 3]);
+                }
+            }
+            // row maximum over the 64-key tile (line 7): own half, then the other half's
+            const bool need_mask = (args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N);
+            if (need_mask) {                                   // masked scores become -inf: exp gives exact zeros
+#pragma unroll
+                for (int i = 0; i < KPT; ++i) p[i] = (kbase + i > key_lim) ? -INFINITY : p[i];
+            }
+            float mx;
+            {
+                float t4[KPT / 4];
+#pragma unroll
+                for (int i = 0; i < KPT / 4; ++i) t4[i] = fmaxf(max3(p[4 * i], p[4 * i + 1], p[4 * i + 2]), p[4 * i + 3]);
+#pragma unroll
+                for (int w = KPT / 8; w >= 1; w >>= 1)
+#pragma unroll
+                    for (int i = 0; i < w; ++i) t4[i] = fmaxf(t4[i], t4[i + w]);
+                mx = t4[0];
+            }
+            xmax[(par * 2 + kq) * 128 + r_loc] = mx;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(xbar);
+            if (!wait256(xbar, par, abort_flag)) { fail(9); ok = false; break; }
+            mx = fmaxf(mx, xmax[(par * 2 + (kq ^ 1)) * 128 + r_loc]);   // the tile is one 64-key group: row max = group max
+
+            const float m_new = fmaxf(m_run, f16_round(mx * args.c0));
+            float rsc = 1.f;
+            if (jt > 0 && m_new != m_run) rsc = f16_round(ex2_approx((m_run - m_new) * LOG2E));
+            m_run = m_new;
+            const float mL = m_run * LOG2E;
+            const float A = p_of_score(mx, args.c1, mL);       // = max of P over the group (monotone map)
+
+            // P = exp(S - m) in FP16 (line 9), P-hat = HIF4(P) (line 10)
+            uint8_t* dc = nullptr;
+            float* ds = nullptr;
+            if (DBG && dbg_slot >= 0 && row < N && kbase < N) {
+                const size_t r_idx = (size_t)dbg_slot * 128 + r_loc;
+                if (args.dbg.p_codes) dc = args.dbg.p_codes + r_idx * N + kbase;
+                if (args.dbg.p_step) ds = args.dbg.p_step + r_idx * (N / 4) + kbase / 4;
+            }
+            uint32_t w[NU * 4];
+            const PQuantConst qc = p_quant_const(args.c1, mL, A);
+            exp_quantize_units<NU, 0, NU, DBG>(p, qc, A == 0.f, w, dc, ds);
+            // the P-hat columns and [O | l] are free once PV(jt-1) has completed (every warp observes
+            // every phase of that barrier, in order)
+            if (jt > 0) {
+                if (!wait256(bar(BAR_PV), par ^ 1u, abort_flag)) { fail(10); ok = false; break; }
+                tc_fence_after();
+            }
+            tmem_st16(t_lane + P_COL + kq * (KPT / 2), w);
+            // rescale history (line 8): each half of the row's threads owns 136 of the 272 columns
+            if (__any_sync(0xffffffffu, rsc != 1.f)) {
+                constexpr int CW = O_COLS / KS;                // 136
+                const uint32_t t_o = t_lane + kq * CW;
+                const uint64_t rr = pack2(rsc, rsc);
+#pragma unroll
+                for (int cc = 0; cc < CW / 32; ++cc) {
+                    uint32_t r[32];
+                    tmem_ld32(t_o + cc * 32, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float x0, x1;
+                        unpack2(mul2(pack2(__uint_as_float(r[i]), __uint_as_float(r[i + 1])), rr), x0, x1);
+                        r[i] = __float_as_uint(x0);
+                        r[i + 1] = __float_as_uint(x1);
+                    }
+                    tmem_st32(t_o + cc * 32, r);
+                }
+#pragma unroll
+                for (int cc = 0; cc < (CW % 32) / 4; ++cc) {
+                    uint32_t r[4];
+                    tmem_ld4(t_o + (CW / 32) * 32 + cc * 4, r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * rsc);
+                    tmem_st4(t_o + (CW / 32) * 32 + cc * 4, r);
+                }
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(BAR_PF));
+        }
+
+        // finalize: out = O / l with l rounded to FP16 (line 13); half kq writes channels 128*kq..
+        if (ok && wait256(bar(BAR_PV), (uint32_t)(n_tiles - 1) & 1u, abort_flag)) {
+            tc_fence_after();
+            uint32_t lr[4];
+            tmem_ld4(t_lane + D, lr);
+            tmem_wait_ld();
+            const float ell = __uint_as_float(lr[0]);
+            const float l16 = f16_round(ell);
+            if (DBG && dbg_slot >= 0 && row < N && kq == 0) {
+                if (args.dbg.l_out) args.dbg.l_out[dbg_slot * 128 + r_loc] = ell;
+                if (args.dbg.m_out) args.dbg.m_out[dbg_slot * 128 + r_loc] = m_run;
+            }
+            const size_t orow = ((size_t)bh_q * N + row) * D + kq * 128;
+#pragma unroll
+            for (int cc = 0; cc < 4; ++cc) {
+                uint32_t r[32];
+                tmem_ld32(t_lane + kq * 128 + cc * 32, r);
+                tmem_wait_ld();
+                if (row < N) {
+                    float o[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) o[i] = __fdiv_rn(__uint_as_float(r[i]), l16);
+                    if (args.out_dtype == HIFA4_F32) {
+                        float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.out) + orow + cc * 32);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+                    } else {
+                        uint32_t w[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            if (args.out_dtype == HIFA4_F16) {
+                                __half2 t = __floats2half2_rn(o[2 * i], o[2 * i + 1]);
+                                w[i] = *reinterpret_cast<uint32_t*>(&t);
+                            } else {
+                                __nv_bfloat162 t = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+                                w[i] = *reinterpret_cast<uint32_t*>(&t);
+                            }
+                        }
+                        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(args.out) + orow + cc * 32);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+                    }
+                }
+            }
+        } else if (ok) {
+            fail(11);
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == W_MMA) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
+}
+
+template <bool DBG>
+static int launch_ws256(const hifa4_shape& sh, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                        const AttnArgs& args, cudaStream_t st)
+{
+    auto kern = attention_fwd_ws256_kernel<DBG>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ws256::SMEM_BYTES) != cudaSuccess)
+            return HIFA4_ERR_CUDA;
+        attr_set = true;
+    }
+    dim3 grid((unsigned)(((sh.N + 127) / 128) * sh.Hq * sh.B));
+    kern<<<grid, ws256::THREADS, ws256::SMEM_BYTES, st>>>(mq, mk, mv, args);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? HIFA4_OK : HIFA4_ERR_CUDA;
+}
+
+int launch_attention_ws256(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
+{
+    CUtensorMap mq, mk, mv;
+    if (!make_bf16_map(&mq, qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, ws256::D, 128)) return HIFA4_ERR_CUDA;
+    if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, ws256::D, ws256::BC)) return HIFA4_ERR_CUDA;
+    if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, ws256::D, sh.N, ws256::D)) return HIFA4_ERR_CUDA;
+    return args.dbg.n_blocks > 0 ? launch_ws256<true>(sh, mq, mk, mv, args, st)
+                                 : launch_ws256<false>(sh, mq, mk, mv, args, st);
+}
+
+}  // namespace hifa4
