@@ -200,6 +200,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--workload", default="C2", help="C2 (headline), C3, C4, C5 or C5@<N>")
     ap.add_argument("--noncausal", action="store_true")
+    ap.add_argument("--Bc", type=int, default=0, help="key-tile width (default: the configuration's, 64)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -215,8 +216,8 @@ def main():
         over["N"] = int(n_over)
     if args.noncausal:
         over["causal"] = False
-    if name == "C4":
-        over.setdefault("Bc", 64)          # d = 256 is built with 64-key tiles
+    if args.Bc:
+        over["Bc"] = args.Bc
     cfg = synth.config(name, **over)
 
     if args.impl == "reference":

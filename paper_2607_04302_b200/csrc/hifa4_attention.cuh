@@ -275,7 +275,7 @@ bool make_bf16_map(CUtensorMap* m, void* base, uint64_t heads, uint64_t rows, ui
 // Warp-specialised kernel for d = 128, Bc = 128 (hifa4_attention_ws.cu).
 int launch_attention_ws(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st);
 
-// Warp-specialised kernel for d = 256, Bc = 64 (hifa4_attention_ws256.cu).
-int launch_attention_ws256(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st);
+// Warp-specialised kernels for Bc = 64, d = 128 or 256 (hifa4_attention_ws64.cu).
+int launch_attention_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st);
 
 }  // namespace hifa4

@@ -1,4 +1,4 @@
-// Warp-specialised HiFA4 attention forward for d = 256, Bc = 64 (Algorithm 1 lines 4-13).
+// Warp-specialised HiFA4 attention forward for Bc = 64 (Algorithm 1 lines 4-13), d = 128 or 256.
 //
 // One CTA = 128 query rows of one (batch, query head), 10 warps:
 //   warps 0-7  softmax / quantize: warp w owns rows 32*(w%4).. of the tile and keys 32*(w/4).. of
@@ -6,40 +6,53 @@
 //              threads of a row exchange their partial score maxima through shared memory
 //   warp 8     TMA producer: Q once, then K and V^T tiles through two-stage rings
 //   warp 9     tcgen05 issuer
-// Tensor memory (512 columns): [O | l] in 0..271 (256 channels by one N = 256 MMA, the ones block by
-// an N = 16 MMA on the same A operand), the Q-hat image in 272..399, one S buffer of 64 columns at
-// 400 and the BF16 image of P-hat in 464..495.  With d = 256 there is no room for a second S buffer,
-// so S is released early instead: the softmax warps pull S(j) into registers and signal it free, and
-// S(j+1) = Q K^T runs on the tensor pipe while they work on tile j; P-hat lives in its own columns.
-// Both GEMMs take their A operand from tensor memory and only K, V^T (with its rows of ones) from
-// shared memory.  Every wait is bounded (see hifa4_attention_ws.cu for the failure protocol).
+// S has a single buffer that is released early: the softmax warps pull S(j) into registers and
+// signal it free, and S(j+1) = Q K^T runs on the tensor pipe while they work on tile j; the BF16
+// image of P-hat has its own tensor-memory columns and is the A operand of the PV MMA.
+//   d = 256: 512 tensor-memory columns: [O | l] 0..271 (an N = 256 MMA for the channels, an N = 16
+//            MMA on the same A operand for the ones block), Q-hat image 272..399 (A operand of
+//            Q K^T from tensor memory), S 400..463, P-hat 464..495.  One CTA per SM.
+//   d = 128: 256 tensor-memory columns: [O | l] 0..143 (one N = 144 MMA), S 144..207, P-hat
+//            208..239; Q-hat stays in shared memory (SS-form Q K^T).  101 KB of shared memory and
+//            <= 102 registers, so two CTAs share an SM and fill each other's synchronisation gaps.
+// Every wait is bounded (see hifa4_attention_ws.cu for the failure protocol).
 #include "hifa4_attention.cuh"
 
 namespace hifa4 {
 
-namespace ws256 {
-constexpr int D = 256, BC = 64, STAGES = 2, KS = 2;
-constexpr int NSW = 4 * KS, THREADS = (NSW + 2) * 32, W_TMA = NSW, W_MMA = NSW + 1;
-constexpr int KPT = BC / KS, NU = KPT / 8;          // 32 keys = 4 level-2 units per thread and tile
-constexpr int Q_BYTES = 4 * 16384;                  // four 64-channel sub-tiles of 128 rows
-constexpr int K_SUB = BC * 128;                     // 64 keys x 64 channels
-constexpr int K_STAGE = 4 * K_SUB;
-constexpr int V_STAGE = (D + 16) * 128;             // 256 rows of V^T + 16 rows of ones, 64 keys wide
-constexpr int Q_OFF = 0;
-constexpr int K_OFF = Q_OFF + Q_BYTES;
-constexpr int V_OFF = K_OFF + STAGES * K_STAGE;
-constexpr int MISC_OFF = V_OFF + STAGES * V_STAGE;
-constexpr int XCHG_OFF = MISC_OFF + 256;            // partial row maxima [2 parities][2 splits][128 rows]
-constexpr int SMEM_BYTES = XCHG_OFF + 2 * 2 * 128 * 4 + 1024;
-constexpr int O_COLS = D + 16, QT_COL = 272, S_COL = 400, P_COL = 464, TMEM_COLS = 512;
+template <int D_>
+struct WS64 {
+    static constexpr int D = D_, BC = 64, STAGES = 2, KS = 2;
+    static constexpr int NSW = 4 * KS, THREADS = (NSW + 2) * 32, W_TMA = NSW, W_MMA = NSW + 1;
+    static constexpr int KPT = BC / KS, NU = KPT / 8;       // 32 keys = 4 level-2 units per thread and tile
+    static constexpr int QSUB = D / 64;                     // 64-channel sub-tiles of Q and K
+    static constexpr int Q_BYTES = QSUB * 16384;
+    static constexpr int K_SUB = BC * 128;                  // 64 keys x 64 channels
+    static constexpr int K_STAGE = QSUB * K_SUB;
+    static constexpr int V_STAGE = (D + 16) * 128;          // D rows of V^T + 16 rows of ones, 64 keys wide
+    static constexpr int Q_OFF = 0;
+    static constexpr int K_OFF = Q_OFF + Q_BYTES;
+    static constexpr int V_OFF = K_OFF + STAGES * K_STAGE;
+    static constexpr int MISC_OFF = V_OFF + STAGES * V_STAGE;
+    static constexpr int XCHG_OFF = MISC_OFF + 256;         // partial row maxima [2 parities][2 splits][128 rows]
+    static constexpr int SMEM_BYTES = XCHG_OFF + 2 * 2 * 128 * 4 + 1024;
+    static constexpr int O_COLS = D + 16;
+    static constexpr bool Q_IN_TMEM = (D == 256);
+    static constexpr int QT_COL = 272;                      // d = 256 only
+    static constexpr int S_COL = (D == 256) ? 400 : 144;
+    static constexpr int P_COL = S_COL + 64;
+    static constexpr int TMEM_COLS = (D == 256) ? 512 : 256;
+    static constexpr int CTAS_PER_SM = (D == 256) ? 1 : 2;
+};
+namespace ws64 {
 enum { BAR_Q = 0, BAR_KF = 1, BAR_KE = 3, BAR_VF = 5, BAR_VE = 7, BAR_SF = 9, BAR_SFREE = 10, BAR_PF = 11,
        BAR_PV = 12, BAR_X = 13, BAR_QT = 17, N_BARS = 18 };
 constexpr uint32_t WAIT_POLLS = 1u << 20;
-}  // namespace ws256
+}  // namespace ws64
 
-static __device__ __forceinline__ bool wait256(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+static __device__ __forceinline__ bool wait64(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
-    for (uint32_t i = 0; i < ws256::WAIT_POLLS / 64; ++i) {
+    for (uint32_t i = 0; i < ws64::WAIT_POLLS / 64; ++i) {
 #pragma unroll 1
         for (int j = 0; j < 64; ++j)
             if (mbar_try_wait(bar, parity)) return true;
@@ -48,23 +61,28 @@ static __device__ __forceinline__ bool wait256(uint32_t bar, uint32_t parity, vo
     return false;
 }
 
-template <bool DBG>
-__global__ void __launch_bounds__(ws256::THREADS, 1)
-attention_fwd_ws256_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+template <int DH, bool DBG>
+__global__ void __launch_bounds__(WS64<DH>::THREADS, WS64<DH>::CTAS_PER_SM)
+attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                            const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnArgs args)
 {
-    using namespace ws256;
+    using namespace ws64;
+    using C = WS64<DH>;
+    constexpr int D = C::D, BC = C::BC, STAGES = C::STAGES, KS = C::KS, NSW = C::NSW, THREADS = C::THREADS;
+    constexpr int W_TMA = C::W_TMA, W_MMA = C::W_MMA, KPT = C::KPT, NU = C::NU, QSUB = C::QSUB;
+    constexpr int Q_BYTES = C::Q_BYTES, K_SUB = C::K_SUB, K_STAGE = C::K_STAGE, V_STAGE = C::V_STAGE;
+    constexpr int O_COLS = C::O_COLS, QT_COL = C::QT_COL, S_COL = C::S_COL, P_COL = C::P_COL, TMEM_COLS = C::TMEM_COLS;
     if (args.d_status && *reinterpret_cast<volatile int*>(args.d_status) != 0) return;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    const uint32_t q_s = smem_base + Q_OFF, k_s = smem_base + K_OFF, v_s = smem_base + V_OFF,
-                   bars = smem_base + MISC_OFF;
+    const uint32_t q_s = smem_base + C::Q_OFF, k_s = smem_base + C::K_OFF, v_s = smem_base + C::V_OFF,
+                   bars = smem_base + C::MISC_OFF;
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + MISC_OFF + 8 * N_BARS);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + MISC_OFF + 8 * N_BARS + 8);
-    float* xmax = reinterpret_cast<float*>(smem_gen + XCHG_OFF);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + C::MISC_OFF + 8 * N_BARS);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + C::MISC_OFF + 8 * N_BARS + 8);
+    float* xmax = reinterpret_cast<float*>(smem_gen + C::XCHG_OFF);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int N = args.N;
@@ -115,17 +133,17 @@ attention_fwd_ws256_kernel(const __grid_constant__ CUtensorMap tmap_q, const __g
         if (lane == 0) {
             mbar_expect_tx(bar(BAR_Q), Q_BYTES);
 #pragma unroll
-            for (int s = 0; s < 4; ++s) tma_load_3d(q_s + s * 16384, &tmap_q, bar(BAR_Q), 64 * s, q0, bh_q);
+            for (int s = 0; s < QSUB; ++s) tma_load_3d(q_s + s * 16384, &tmap_q, bar(BAR_Q), 64 * s, q0, bh_q);
             for (int jt = 0; jt < n_tiles; ++jt) {
                 const int st = jt & 1;
                 const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
                 const int j0 = jt * BC;
-                if (!wait256(bar(BAR_KE + st), ph ^ 1u, abort_flag)) { fail(1); break; }
+                if (!wait64(bar(BAR_KE + st), ph ^ 1u, abort_flag)) { fail(1); break; }
                 mbar_expect_tx(bar(BAR_KF + st), K_STAGE);
 #pragma unroll
-                for (int s = 0; s < 4; ++s)
+                for (int s = 0; s < QSUB; ++s)
                     tma_load_3d(k_s + st * K_STAGE + s * K_SUB, &tmap_k, bar(BAR_KF + st), 64 * s, j0, bh_kv);
-                if (!wait256(bar(BAR_VE + st), ph ^ 1u, abort_flag)) { fail(2); break; }
+                if (!wait64(bar(BAR_VE + st), ph ^ 1u, abort_flag)) { fail(2); break; }
                 mbar_expect_tx(bar(BAR_VF + st), D * 128);
                 tma_load_3d(v_s + st * V_STAGE, &tmap_v, bar(BAR_VF + st), j0, 0, bh_kv);
             }
@@ -133,45 +151,48 @@ attention_fwd_ws256_kernel(const __grid_constant__ CUtensorMap tmap_q, const __g
     } else if (warp == W_MMA) {
         // ------------------------------------------------------------------ tcgen05 issuer
         constexpr uint32_t idesc_s = umma_idesc_bf16(128, BC);
-        constexpr uint32_t idesc_o = umma_idesc_bf16(128, 256);
+        constexpr uint32_t idesc_o = umma_idesc_bf16(128, D == 256 ? 256 : O_COLS);
         constexpr uint32_t idesc_l = umma_idesc_bf16(128, 16);
         const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
-        const uint32_t k_lo = umma_desc_lo(k_s), v_lo = umma_desc_lo(v_s);
+        const uint32_t q_lo = umma_desc_lo(q_s), k_lo = umma_desc_lo(k_s), v_lo = umma_desc_lo(v_s);
         const bool leader = elect_one();
         bool ok = true;
-        auto issue_qk = [&](int jt) {                     // S(jt) from K stage jt % 2 (16 steps of 16 channels)
+        auto issue_qk = [&](int jt) {                     // S(jt) from K stage jt % 2 (D / 16 steps of 16 channels)
             const uint32_t b0 = k_lo + (jt & 1) * (K_STAGE >> 4);
             if (leader) {
 #pragma unroll
-                for (int kk = 0; kk < 16; ++kk)
-                    umma_bf16_ts_lo(tm + S_COL, tm + QT_COL + kk * 8, b0 + (kk >> 2) * (K_SUB >> 4) + (kk & 3) * 2,
-                                    idesc_s, kk ? 1u : 0u);
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t kb = b0 + (kk >> 2) * (K_SUB >> 4) + (kk & 3) * 2;
+                    if constexpr (C::Q_IN_TMEM) umma_bf16_ts_lo(tm + S_COL, tm + QT_COL + kk * 8, kb, idesc_s, kk ? 1u : 0u);
+                    else umma_bf16_ss_lo(tm + S_COL, q_lo + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2, kb, idesc_s, kk ? 1u : 0u);
+                }
                 umma_commit(bar(BAR_SF));
                 umma_commit(bar(BAR_KE + (jt & 1)));
             }
             __syncwarp();
         };
-        ok = wait256(bar(BAR_QT), 0, abort_flag) && wait256(bar(BAR_KF), 0, abort_flag);
+        ok = wait64(bar(C::Q_IN_TMEM ? BAR_QT : BAR_Q), 0, abort_flag) && wait64(bar(BAR_KF), 0, abort_flag);
         if (ok) { tc_fence_after(); issue_qk(0); } else if (leader) fail(3);
         for (int jt = 0; ok && jt < n_tiles; ++jt) {
             const int st = jt & 1;
             const uint32_t ph = (uint32_t)(jt >> 1) & 1u, par = (uint32_t)jt & 1u;
             if (jt + 1 < n_tiles) {                       // S(jt+1) as soon as S(jt) sits in registers
-                if (!wait256(bar(BAR_KF + (st ^ 1)), (uint32_t)((jt + 1) >> 1) & 1u, abort_flag)) { if (leader) fail(4); break; }
-                if (!wait256(bar(BAR_SFREE), par, abort_flag)) { if (leader) fail(5); break; }
+                if (!wait64(bar(BAR_KF + (st ^ 1)), (uint32_t)((jt + 1) >> 1) & 1u, abort_flag)) { if (leader) fail(4); break; }
+                if (!wait64(bar(BAR_SFREE), par, abort_flag)) { if (leader) fail(5); break; }
                 tc_fence_after();
                 issue_qk(jt + 1);
             }
-            if (!wait256(bar(BAR_VF + st), ph, abort_flag)) { if (leader) fail(6); break; }
-            if (!wait256(bar(BAR_PF), par, abort_flag)) { if (leader) fail(7); break; }
+            if (!wait64(bar(BAR_VF + st), ph, abort_flag)) { if (leader) fail(6); break; }
+            if (!wait64(bar(BAR_PF), par, abort_flag)) { if (leader) fail(7); break; }
             tc_fence_after();
             const uint32_t b0 = v_lo + st * (V_STAGE >> 4);
             const uint32_t acc0 = jt > 0 ? 1u : 0u;
             if (leader) {
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {            // 16 keys per step; channels, then the ones block
+                for (int kk = 0; kk < 4; ++kk) {            // 16 keys per step; channels (+ ones block)
                     umma_bf16_ts_lo(tm, tm + P_COL + kk * 8, b0 + kk * 2, idesc_o, kk ? 1u : acc0);
-                    umma_bf16_ts_lo(tm + 256, tm + P_COL + kk * 8, b0 + ((D * 128) >> 4) + kk * 2, idesc_l, kk ? 1u : acc0);
+                    if constexpr (D == 256)                  // N = 272 does not exist: the ones block separately
+                        umma_bf16_ts_lo(tm + 256, tm + P_COL + kk * 8, b0 + ((D * 128) >> 4) + kk * 2, idesc_l, kk ? 1u : acc0);
                 }
                 umma_commit(bar(BAR_PV));
                 umma_commit(bar(BAR_VE + st));
@@ -196,33 +217,36 @@ attention_fwd_ws256_kernel(const __grid_constant__ CUtensorMap tmap_q, const __g
         float m_run = -INFINITY;
         bool ok = true;
 
-        // Q-hat image: shared memory (swizzled TMA tiles) -> tensor memory; this thread moves 128
-        // channels of its row = 64 columns of packed BF16 pairs.
-        if (wait256(bar(BAR_Q), 0, abort_flag)) {
-            const int sw = r_loc & 7;
+        // d = 256: Q-hat image, shared memory (swizzled TMA tiles) -> tensor memory; this thread moves 128
+        // channels of its row = 64 columns of packed BF16 pairs.  (d = 128: the issuer waits for the
+        // Q load itself.)
+        if constexpr (C::Q_IN_TMEM) {
+            if (wait64(bar(BAR_Q), 0, abort_flag)) {
+                const int sw = r_loc & 7;
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t qw[32];
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t qw[32];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const int chunk = kq * 16 + half * 8 + c;          // 16-byte chunk of the 512-byte row
-                    const uint32_t a = q_s + (chunk >> 3) * 16384 + (r_loc >> 3) * 1024 + sw * 128 + (((chunk & 7) ^ sw) << 4);
-                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                                 : "=r"(qw[4 * c]), "=r"(qw[4 * c + 1]), "=r"(qw[4 * c + 2]), "=r"(qw[4 * c + 3]) : "r"(a));
+                    for (int c = 0; c < 8; ++c) {
+                        const int chunk = kq * 16 + half * 8 + c;      // 16-byte chunk of the 512-byte row
+                        const uint32_t a = q_s + (chunk >> 3) * 16384 + (r_loc >> 3) * 1024 + sw * 128 + (((chunk & 7) ^ sw) << 4);
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                     : "=r"(qw[4 * c]), "=r"(qw[4 * c + 1]), "=r"(qw[4 * c + 2]), "=r"(qw[4 * c + 3]) : "r"(a));
+                    }
+                    tmem_st32(t_lane + QT_COL + kq * 64 + half * 32, qw);
                 }
-                tmem_st32(t_lane + QT_COL + kq * 64 + half * 32, qw);
-            }
-            tmem_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_QT));
-        } else { fail(13); ok = false; }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(BAR_QT));
+            } else { fail(13); ok = false; }
+        }
 
         for (int jt = 0; ok && jt < n_tiles; ++jt) {
             const int j0 = jt * BC;
             const uint32_t par = (uint32_t)jt & 1u;
             const int kbase = j0 + kq * KPT;
-            if (!wait256(bar(BAR_SF), par, abort_flag)) { fail(8); ok = false; break; }
+            if (!wait64(bar(BAR_SF), par, abort_flag)) { fail(8); ok = false; break; }
             tc_fence_after();
             float p[KPT];
             {
@@ -267,7 +291,7 @@ attention_fwd_ws256_kernel(const __grid_constant__ CUtensorMap tmap_q, const __g
             xmax[(par * 2 + kq) * 128 + r_loc] = mx;
             __syncwarp();
             if (lane == 0) mbar_arrive(xbar);
-            if (!wait256(xbar, par, abort_flag)) { fail(9); ok = false; break; }
+            if (!wait64(xbar, par, abort_flag)) { fail(9); ok = false; break; }
             mx = fmaxf(mx, xmax[(par * 2 + (kq ^ 1)) * 128 + r_loc]);   // the tile is one 64-key group: row max = group max
 
             const float m_new = fmaxf(m_run, f16_round(mx * args.c0));
@@ -291,13 +315,13 @@ attention_fwd_ws256_kernel(const __grid_constant__ CUtensorMap tmap_q, const __g
             // the P-hat columns and [O | l] are free once PV(jt-1) has completed (every warp observes
             // every phase of that barrier, in order)
             if (jt > 0) {
-                if (!wait256(bar(BAR_PV), par ^ 1u, abort_flag)) { fail(10); ok = false; break; }
+                if (!wait64(bar(BAR_PV), par ^ 1u, abort_flag)) { fail(10); ok = false; break; }
                 tc_fence_after();
             }
             tmem_st16(t_lane + P_COL + kq * (KPT / 2), w);
-            // rescale history (line 8): each half of the row's threads owns 136 of the 272 columns
+            // rescale history (line 8): each half of the row's threads owns half of the d + 16 columns
             if (__any_sync(0xffffffffu, rsc != 1.f)) {
-                constexpr int CW = O_COLS / KS;                // 136
+                constexpr int CW = O_COLS / KS;                // 136 or 72
                 const uint32_t t_o = t_lane + kq * CW;
                 const uint64_t rr = pack2(rsc, rsc);
 #pragma unroll
@@ -330,8 +354,8 @@ attention_fwd_ws256_kernel(const __grid_constant__ CUtensorMap tmap_q, const __g
             if (lane == 0) mbar_arrive(bar(BAR_PF));
         }
 
-        // finalize: out = O / l with l rounded to FP16 (line 13); half kq writes channels 128*kq..
-        if (ok && wait256(bar(BAR_PV), (uint32_t)(n_tiles - 1) & 1u, abort_flag)) {
+        // finalize: out = O / l with l rounded to FP16 (line 13); half kq writes channels (d/2)*kq..
+        if (ok && wait64(bar(BAR_PV), (uint32_t)(n_tiles - 1) & 1u, abort_flag)) {
             tc_fence_after();
             uint32_t lr[4];
             tmem_ld4(t_lane + D, lr);
@@ -342,11 +366,11 @@ attention_fwd_ws256_kernel(const __grid_constant__ CUtensorMap tmap_q, const __g
                 if (args.dbg.l_out) args.dbg.l_out[dbg_slot * 128 + r_loc] = ell;
                 if (args.dbg.m_out) args.dbg.m_out[dbg_slot * 128 + r_loc] = m_run;
             }
-            const size_t orow = ((size_t)bh_q * N + row) * D + kq * 128;
+            const size_t orow = ((size_t)bh_q * N + row) * D + kq * (D / 2);
 #pragma unroll
-            for (int cc = 0; cc < 4; ++cc) {
+            for (int cc = 0; cc < D / 64; ++cc) {
                 uint32_t r[32];
-                tmem_ld32(t_lane + kq * 128 + cc * 32, r);
+                tmem_ld32(t_lane + kq * (D / 2) + cc * 32, r);
                 tmem_wait_ld();
                 if (row < N) {
                     float o[32];
@@ -384,31 +408,33 @@ attention_fwd_ws256_kernel(const __grid_constant__ CUtensorMap tmap_q, const __g
     if (warp == W_MMA) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
 }
 
-template <bool DBG>
-static int launch_ws256(const hifa4_shape& sh, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                        const AttnArgs& args, cudaStream_t st)
+template <int DH, bool DBG>
+static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
-    auto kern = attention_fwd_ws256_kernel<DBG>;
+    using C = WS64<DH>;
+    CUtensorMap mq, mk, mv;
+    if (!make_bf16_map(&mq, qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, DH, 128)) return HIFA4_ERR_CUDA;
+    if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, DH, C::BC)) return HIFA4_ERR_CUDA;
+    if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, DH, sh.N, DH)) return HIFA4_ERR_CUDA;
+    auto kern = attention_fwd_ws64_kernel<DH, DBG>;
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ws256::SMEM_BYTES) != cudaSuccess)
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
             return HIFA4_ERR_CUDA;
         attr_set = true;
     }
     dim3 grid((unsigned)(((sh.N + 127) / 128) * sh.Hq * sh.B));
-    kern<<<grid, ws256::THREADS, ws256::SMEM_BYTES, st>>>(mq, mk, mv, args);
+    kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mq, mk, mv, args);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? HIFA4_OK : HIFA4_ERR_CUDA;
 }
 
-int launch_attention_ws256(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
+int launch_attention_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
-    CUtensorMap mq, mk, mv;
-    if (!make_bf16_map(&mq, qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, ws256::D, 128)) return HIFA4_ERR_CUDA;
-    if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, ws256::D, ws256::BC)) return HIFA4_ERR_CUDA;
-    if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, ws256::D, sh.N, ws256::D)) return HIFA4_ERR_CUDA;
-    return args.dbg.n_blocks > 0 ? launch_ws256<true>(sh, mq, mk, mv, args, st)
-                                 : launch_ws256<false>(sh, mq, mk, mv, args, st);
+    const bool dbg = args.dbg.n_blocks > 0;
+    if (sh.d == 256) return dbg ? launch_ws64<256, true>(sh, qkv, args, st) : launch_ws64<256, false>(sh, qkv, args, st);
+    if (sh.d == 128) return dbg ? launch_ws64<128, true>(sh, qkv, args, st) : launch_ws64<128, false>(sh, qkv, args, st);
+    return HIFA4_ERR_UNSUPPORTED;
 }
 
 }  // namespace hifa4

@@ -25,7 +25,7 @@ class Config:
     outlier_gain: float
     smooth_mode: int        # 0 bypass, 1 strong (alpha .5), 2 mild (alpha .25)
     Br: int
-    Bc: int
+    Bc: int              # key-tile width of the online softmax (part of the result); 64 is the fastest path
     seed: int = 0
     fixed_outliers: tuple = ()   # explicit channel list (same for every head)
     cal_samples: int = 4
@@ -37,15 +37,15 @@ CONFIGS = {
     "C1": Config("C1-tiny", 1, 1, 1, 128, 128, False, "fp16", 4, 20.0, 1, 64, 64,
                  fixed_outliers=(3, 17, 64, 101), cal_samples=4, cal_tokens=128),
     # Qwen3-8B-shaped GQA prefill, 4 of 128 K channels x20 per KV head
-    "C2": Config("C2-qwen3-8b-4k", 1, 32, 8, 4096, 128, True, "bf16", 4, 20.0, 1, 128, 128,
+    "C2": Config("C2-qwen3-8b-4k", 1, 32, 8, 4096, 128, True, "bf16", 4, 20.0, 1, 128, 64,
                  cal_samples=32, cal_tokens=1024),
     # LLaMA3.1-8B-shaped, no outliers, smoothing bypassed
-    "C3": Config("C3-llama31-8b-8k", 1, 32, 8, 8192, 128, True, "bf16", 0, 1.0, 0, 128, 128),
+    "C3": Config("C3-llama31-8b-8k", 1, 32, 8, 8192, 128, True, "bf16", 0, 1.0, 0, 128, 64),
     # Gemma2-9B-shaped, d=256, 2 of 256 channels x8, mild smoothing
-    "C4": Config("C4-gemma2-9b-8k", 1, 16, 8, 8192, 256, True, "bf16", 2, 8.0, 2, 128, 128,
+    "C4": Config("C4-gemma2-9b-8k", 1, 16, 8, 8192, 256, True, "bf16", 2, 8.0, 2, 128, 64,
                  cal_samples=8, cal_tokens=1024),
     # sequence sweep base point (N and causal are overridden by the caller)
-    "C5": Config("C5-sweep", 4, 32, 8, 1024, 128, True, "bf16", 4, 20.0, 1, 128, 128,
+    "C5": Config("C5-sweep", 4, 32, 8, 1024, 128, True, "bf16", 4, 20.0, 1, 128, 64,
                  cal_samples=8, cal_tokens=1024),
 }
 

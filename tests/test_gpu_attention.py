@@ -33,16 +33,21 @@ def test_tiny_config(hb, par):
 
 
 SMALL = {
-    "d128-bc128-causal-gqa": synth.config("C2", N=512, Hq=4, Hkv=2, cal_samples=4, cal_tokens=128),
+    "d128-bc128-causal-gqa": synth.config("C2", N=512, Hq=4, Hkv=2, Bc=128, cal_samples=4, cal_tokens=128),
+    "d128-bc64-causal-gqa": synth.config("C2", N=512, Hq=4, Hkv=2, cal_samples=4, cal_tokens=128),
     "d128-bc64-causal": synth.config("C2", N=384, Hq=2, Hkv=1, Bc=64, cal_samples=4, cal_tokens=128),
-    "d128-bc128-noncausal": synth.config("C2", N=256, Hq=2, Hkv=2, causal=False, cal_samples=4, cal_tokens=128),
-    "d128-ragged-n": synth.config("C2", N=320, Hq=2, Hkv=1, cal_samples=4, cal_tokens=128),
-    "d128-ragged-noncausal": synth.config("C3", N=192, Hq=1, Hkv=1, causal=False),
-    "d64-bc128": synth.config("C3", N=256, Hq=2, Hkv=1, d=64),
+    "d128-bc128-noncausal": synth.config("C2", N=256, Hq=2, Hkv=2, Bc=128, causal=False, cal_samples=4, cal_tokens=128),
+    "d128-ragged-n": synth.config("C2", N=320, Hq=2, Hkv=1, Bc=128, cal_samples=4, cal_tokens=128),
+    "d128-bc64-ragged-n": synth.config("C2", N=320, Hq=2, Hkv=1, cal_samples=4, cal_tokens=128),
+    "d128-ragged-noncausal": synth.config("C3", N=192, Hq=1, Hkv=1, Bc=128, causal=False),
+    "d128-bc64-noncausal": synth.config("C3", N=192, Hq=1, Hkv=1, causal=False),
+    "d64-bc128": synth.config("C3", N=256, Hq=2, Hkv=1, d=64, Bc=128),
     "d64-bc64-fp16": synth.config("C3", N=256, Hq=2, Hkv=1, d=64, Bc=64, dtype="fp16"),
     "d256-bc64-mild": synth.config("C4", N=256, Hq=2, Hkv=1, Bc=64, cal_samples=3, cal_tokens=64),
-    "batch2": synth.config("C5", B=2, N=256, Hq=4, Hkv=2, cal_samples=2, cal_tokens=64),
-    "n64": synth.config("C3", N=64, Hq=1, Hkv=1),
+    "batch2": synth.config("C5", B=2, N=256, Hq=4, Hkv=2, Bc=128, cal_samples=2, cal_tokens=64),
+    "batch2-bc64": synth.config("C5", B=2, N=256, Hq=4, Hkv=2, cal_samples=2, cal_tokens=64),
+    "n64": synth.config("C3", N=64, Hq=1, Hkv=1, Bc=128),
+    "n64-bc64": synth.config("C3", N=64, Hq=1, Hkv=1),
 }
 
 
@@ -98,15 +103,15 @@ def _sampled_blocks(cfg, heads):
     return [(b, h, t) for b in (0, cfg.B - 1) for h in heads for t in sorted({0, n_qb // 2, n_qb - 1})]
 
 
-@pytest.mark.parametrize("name", ["C2", "C3", "C4"])
-def test_full_size_sampled_blocks(hb, par, name):
-    """Full-size configurations in the launch configuration the benchmark times; the oracle
-    evaluates sampled rows of the first, a middle and the last query block of two heads."""
-    over = dict(Bc=64) if name == "C4" else {}
-    cfg = synth.config(name, cal_samples=4, cal_tokens=256, **over)
+@pytest.mark.parametrize("name,Bc", [("C2", 64), ("C3", 64), ("C4", 64), ("C2", 128), ("C3", 128)])
+def test_full_size_sampled_blocks(hb, par, name, Bc):
+    """Full-size configurations in the launch configuration the benchmark times (Bc = 64) and with
+    the 128-key tiles of the persistent kernel; the oracle evaluates sampled rows of the first, a
+    middle and the last query block of two heads."""
+    cfg = synth.config(name, cal_samples=4, cal_tokens=256, Bc=Bc)
     blocks = sorted(set(_sampled_blocks(cfg, (0, cfg.Hq - 1))))
     res = par.run_case(cfg, DEV, blocks=blocks, check_quant=(name == "C2"), rows_per_block=24)
-    print(par.assert_within_bars(res, name))
+    print(par.assert_within_bars(res, f"{name} Bc={Bc}"))
     out = res["out"]
     assert torch.isfinite(out).all()
 
@@ -120,16 +125,18 @@ def test_sweep_point_sampled(hb, par, causal):
     print(par.assert_within_bars(res, f"C5 N=2048 causal={causal}"))
 
 
-def test_sweep_point_8k_sampled(hb, par):
-    """Configuration 5 at N = 8192 (B = 4, causal): 8192 work items on the persistent kernel."""
-    cfg = synth.config("C5", N=8192, cal_samples=2, cal_tokens=256)
+@pytest.mark.parametrize("Bc", [64, 128])
+def test_sweep_point_8k_sampled(hb, par, Bc):
+    """Configuration 5 at N = 8192 (B = 4, causal): 8192 CTAs of the 64-key kernel, 8192 work items of
+    the persistent 128-key kernel."""
+    cfg = synth.config("C5", N=8192, Bc=Bc, cal_samples=2, cal_tokens=256)
     blocks = [(0, 0, 0), (3, 31, 63), (2, 9, 31), (1, 30, 1)]
     res = par.run_case(cfg, DEV, blocks=blocks, check_quant=False, rows_per_block=12)
     print(par.assert_within_bars(res, "C5 N=8192 causal"))
 
 
-@pytest.mark.parametrize("causal", [True, False])
-def test_largest_sequence_properties(hb, causal):
+@pytest.mark.parametrize("causal,Bc", [(True, 64), (False, 64), (True, 128)])
+def test_largest_sequence_properties(hb, causal, Bc):
     """N = 32768 (the top of the sequence sweep), too large for the oracle: properties that hold at any
     size.  With V constant per channel the output must be that constant's HIF4 value times
     rowsum(P-hat) / FP16(rowsum(P-hat)): numerator and normalizer come from the same P-hat
@@ -142,8 +149,8 @@ def test_largest_sequence_properties(hb, causal):
     v = consts.expand(B, Hkv, N, d).contiguous()
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     qkv = hb.quantize_qkv(q, k, v, d_status=status)
-    out = hb.attention_fwd(qkv, causal, Bc=128, d_status=status)
-    out2 = hb.attention_fwd(qkv, causal, Bc=128, d_status=status)
+    out = hb.attention_fwd(qkv, causal, Bc=Bc, d_status=status)
+    out2 = hb.attention_fwd(qkv, causal, Bc=Bc, d_status=status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert torch.equal(out, out2) and torch.isfinite(out).all()
@@ -155,8 +162,9 @@ def test_largest_sequence_properties(hb, causal):
 
 
 QMEAN = {
-    "qmean-d128-causal-gqa": synth.config("C2", N=512, Hq=4, Hkv=2, cal_samples=4, cal_tokens=128),
-    "qmean-d128-ragged-noncausal": synth.config("C2", N=320, Hq=2, Hkv=1, causal=False, cal_samples=4, cal_tokens=128),
+    "qmean-d128-causal-gqa": synth.config("C2", N=512, Hq=4, Hkv=2, Bc=128, cal_samples=4, cal_tokens=128),
+    "qmean-d128-bc64-causal-gqa": synth.config("C2", N=512, Hq=4, Hkv=2, cal_samples=4, cal_tokens=128),
+    "qmean-d128-ragged-noncausal": synth.config("C2", N=320, Hq=2, Hkv=1, Bc=128, causal=False, cal_samples=4, cal_tokens=128),
     "qmean-tiny-64x64-fp16": synth.config("C1"),
     "qmean-d256-bc64": synth.config("C4", N=256, Hq=2, Hkv=1, Bc=64, cal_samples=3, cal_tokens=64),
 }
