@@ -144,13 +144,8 @@ int hifa4_quantize_qkv(const hifa4_shape* shape, const void* q, const void* k, c
     if ((rc = build_map(shape->Hq, shape->Hkv, shape->q_to_kv, qmap, kmap))) return rc;
     if ((rc = check_arch())) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    const int B = shape->B, N = shape->N, d = shape->d, dt = shape->in_dtype;
-    if (q && launch_quantize_rows(dt, q, s, qmap, B, shape->Hq, N, d, out->q_codes, out->q_meta,
-                                  out->q_mma, out->q_mu, nullptr, st) != cudaSuccess) return HIFA4_ERR_CUDA;
-    if (k && launch_quantize_rows(dt, k, inv_s, kmap, B, shape->Hkv, N, d, out->k_codes, out->k_meta,
-                                  out->k_mma, nullptr, out->k_sum, st) != cudaSuccess) return HIFA4_ERR_CUDA;
-    if (v && launch_quantize_tokens(dt, v, B, shape->Hkv, N, d, out->v_codes, out->v_meta,
-                                    out->v_mma, st) != cudaSuccess) return HIFA4_ERR_CUDA;
+    if (launch_quantize_qkv(shape->in_dtype, *shape, qmap, q, k, v, s, inv_s, *out, st) != cudaSuccess)
+        return HIFA4_ERR_CUDA;
     return HIFA4_OK;
 }
 

@@ -69,13 +69,6 @@ __device__ __forceinline__ void exp2_f16_pair(float t0, float t1, float& e0, flo
         : "=f"(e0), "=f"(e1) : "r"(h2));
 }
 
-__device__ __forceinline__ float max3(float a, float b, float c)
-{
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-
 // Quantize NU*8 consecutive softmax weights of one 64-key HIF4 group (already rounded to FP16,
 // held as floats, all >= 0) and return the BF16 image of P-hat as NU*4 packed words (element 2i
 // in the low half of word i).  A is the maximum of the whole group (the caller combines partial

@@ -10,12 +10,11 @@ struct HeadMap;
 
 void count_launch();
 
-// mu_out: subtract the per-row mean (Q-Mean) and write it; ksum_out: write the per-row channel sum.
-cudaError_t launch_quantize_rows(int dtype, const void* x, const float* scale, const HeadMap& map,
-                                 int B, int H, int N, int d, uint8_t* codes, uint32_t* meta,
-                                 void* img, float* mu_out, float* ksum_out, cudaStream_t st);
-cudaError_t launch_quantize_tokens(int dtype, const void* x, int B, int H, int N, int d,
-                                   uint8_t* codes, uint32_t* meta, void* img, cudaStream_t st);
+// One launch for Q, K and V (null inputs are skipped).  out.q_mu / out.k_sum non-null: Q-Mean
+// (subtract the per-row mean of Q and write it; write the per-row channel sum of K).
+cudaError_t launch_quantize_qkv(int dtype, const hifa4_shape& sh, const HeadMap& qmap, const void* q,
+                                const void* k, const void* v, const float* s, const float* inv_s,
+                                const hifa4_qkv& out, cudaStream_t st);
 cudaError_t launch_absmax(int dtype, const void* x, const HeadMap& map, int S, int H, int Hkv,
                           int Ncal, int d, float* ws, cudaStream_t st);
 cudaError_t launch_smooth_finalize(const float* kmax, const float* qmax, int S, int n, double alpha,

@@ -239,6 +239,13 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
 }
 
 // ------------------------------------------------------------------ packed fp32 pairs
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
 __device__ __forceinline__ uint64_t pack2(float lo, float hi)
 {
     uint64_t r;

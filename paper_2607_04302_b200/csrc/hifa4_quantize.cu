@@ -1,51 +1,77 @@
 // Smooth-QK scaling fused with HIF4 quantization (Algorithm 1 lines 1 and 3) and the
-// calibration reduction behind the Smooth-QK factors (Eq. "sqk").  HBM-bound kernels:
-// 128-bit coalesced loads, one 8-lane team per 64-element group, shuffle reductions.
+// calibration reduction behind the Smooth-QK factors (Eq. "sqk").  Q, K and V are quantized by one
+// launch: 128-bit coalesced loads, one 8-lane team per 64-element group, shuffle reductions,
+// packed f32x2 arithmetic.
 #include "hifa4_internal.h"
 #include "hifa4_device.cuh"
+#include "hifa4_ptx.cuh"
 
 namespace hifa4 {
 
+using namespace ptx;
+
 // One lane owns 8 consecutive elements of a 64-element group = one level-2 unit = two
 // level-3 subgroups; the 8 lanes of a team (aligned inside a warp) own the group.
-// x[8]: values already smoothed and rounded to the input dtype.
-// Returns the packed nibbles; img gets the dequantized values; meta_part gets this lane's
-// OR-contribution (the team leader's includes the scale code).
-__device__ __forceinline__ uint32_t quantize8(const float (&x)[8], int j, float (&img)[8],
-                                              uint32_t& meta_word)
+// x[8]: values already smoothed and rounded to the input dtype.  Returns the packed nibbles; w gets
+// the BF16 image of the dequantized values (element 2i in the low half of word i); meta_word the
+// group's metadata (every lane of the team gets the same word).
+//
+// Arithmetic (all exact; the same scheme as the in-register quantizer of P):
+//   q = RZ(x * RN(4/S))             lands exactly on j + 1/2 on every rounding tie (see e6m2_inv4)
+//   y = q + 1.5 * 2^(23+k)          rounds q to the nearest multiple of 2^k, ties to even:
+//                                   bits(y) - bits(magic) = m, the signed element code under shift k
+//   v = fma(y, S/4, -magic * S/4)   = m * 2^k * S/4, the dequantized value
+// The shift of a subgroup with maximum At is need = max(bits(At) - bits(1.75 S) - 1 + 2^23, 0) >> 23;
+// the pair rule is a = (n0 + n1 + 2) >> 2, k = max(need, a).
+__device__ __forceinline__ uint32_t quantize8(float (&x)[8], int j, uint32_t (&w)[4], uint32_t& meta_word)
 {
-    float a0 = fmaxf(fmaxf(fabsf(x[0]), fabsf(x[1])), fmaxf(fabsf(x[2]), fabsf(x[3])));
-    float a1 = fmaxf(fmaxf(fabsf(x[4]), fabsf(x[5])), fmaxf(fabsf(x[6]), fabsf(x[7])));
+    float a0 = fmaxf(max3(fabsf(x[0]), fabsf(x[1]), fabsf(x[2])), fabsf(x[3]));
+    float a1 = fmaxf(max3(fabsf(x[4]), fabsf(x[5]), fabsf(x[6])), fabsf(x[7]));
     float A = fmaxf(a0, a1);
     A = fmaxf(A, __shfl_xor_sync(0xffffffffu, A, 1));
     A = fmaxf(A, __shfl_xor_sync(0xffffffffu, A, 2));
     A = fmaxf(A, __shfl_xor_sync(0xffffffffu, A, 4));
-    uint32_t nib = 0, part = 0;
-    if (A > 0.f) {
-        int code = e6m2_code_for_max(A);
-        float S = e6m2_value(code);
-        float inv4 = e6m2_inv4(code);
-        int a, b0, b1;
-        hif4_pair_bits(hif4_need(a0, S), hif4_need(a1, S), a, b0, b1);
-        part = ((uint32_t)a << (8 + j)) | ((uint32_t)(b0 | (b1 << 1)) << (16 + 2 * j));
-        if (j == 0) part |= (uint32_t)code;
+    const int code = e6m2_code_for_max(A);                        // A = 0 gives code 0 and an all-zero group
+    const float S = e6m2_value(code);
+    const float top = 7.f * S;
+    if (A > top) {                                                // only above the E6M2 range: saturate
 #pragma unroll
-        for (int w = 0; w < 2; ++w) {
-            int k = a + (w ? b1 : b0);
-            float inv_step = scale_pow2(inv4, -k);
-            float step = scale_pow2(S, k - 2);
+        for (int i = 0; i < 8; ++i) x[i] = fminf(fmaxf(x[i], -top), top);
+        a0 = fminf(a0, top);
+        a1 = fminf(a1, top);
+    }
+    const float inv4 = e6m2_inv4(code);
+    const float S4 = __uint_as_float(__float_as_uint(S) - (2u << 23));
+    const uint64_t inv44 = pack2(inv4, inv4), s44 = pack2(S4, S4);
+    const uint32_t c0_bits = __float_as_uint(-12582912.f * S4);   // -1.5 * 2^23 * S/4
+    const int tadd = (1 << 23) - ((int)__float_as_uint(1.75f * S) + 1);
+    const int n0 = max((int)__float_as_uint(a0) + tadd, 0) >> 23;
+    const int n1 = max((int)__float_as_uint(a1) + tadd, 0) >> 23;
+    const int a = (n0 + n1 + 2) >> 2;
+    const int k0 = max(n0, a), k1 = max(n1, a);
+    uint32_t part = ((uint32_t)a << (8 + j)) | ((uint32_t)((k0 - a) | ((k1 - a) << 1)) << (16 + 2 * j));
+    if (j == 0) part |= (uint32_t)code;
+    uint32_t nib = 0;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                float v = x[4 * w + i];
-                int m = hif4_code(fabsf(v), inv_step);
-                float dq = (float)m * step;
-                img[4 * w + i] = v < 0.f ? -dq : dq;
-                nib |= (uint32_t)(m | ((v < 0.f && m > 0) ? 8 : 0)) << (4 * (4 * w + i));
-            }
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t ks = (uint32_t)(h ? k1 : k0) << 23;
+        const uint32_t magic_bits = 0x4B400000u + ks;
+        const float magic = __uint_as_float(magic_bits), ck = __uint_as_float(c0_bits + ks);
+        const uint64_t mm = pack2(magic, magic), cc = pack2(ck, ck);
+        const uint64_t y01 = add2(mul2_rz(pack2(x[4 * h], x[4 * h + 1]), inv44), mm);
+        const uint64_t y23 = add2(mul2_rz(pack2(x[4 * h + 2], x[4 * h + 3]), inv44), mm);
+        float v0, v1, v2, v3, y[4];
+        unpack2(fma2(y01, s44, cc), v0, v1);
+        unpack2(fma2(y23, s44, cc), v2, v3);
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[2 * h]) : "f"(v1), "f"(v0));
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[2 * h + 1]) : "f"(v3), "f"(v2));
+        unpack2(y01, y[0], y[1]);
+        unpack2(y23, y[2], y[3]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int m = (int)(__float_as_uint(y[i]) - magic_bits);          // signed code
+            nib |= ((uint32_t)abs(m) | ((uint32_t)(m >> 28) & 8u)) << (4 * (4 * h + i));
         }
-    } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) img[i] = 0.f;
     }
     part |= __shfl_xor_sync(0xffffffffu, part, 1);
     part |= __shfl_xor_sync(0xffffffffu, part, 2);
@@ -54,98 +80,177 @@ __device__ __forceinline__ uint32_t quantize8(const float (&x)[8], int j, float 
     return nib;
 }
 
-__device__ __forceinline__ uint4 pack_bf16x8(const float (&v)[8])
-{
-    uint4 o;
-    __nv_bfloat162 t;
-    t = __floats2bfloat162_rn(v[0], v[1]); o.x = *reinterpret_cast<uint32_t*>(&t);
-    t = __floats2bfloat162_rn(v[2], v[3]); o.y = *reinterpret_cast<uint32_t*>(&t);
-    t = __floats2bfloat162_rn(v[4], v[5]); o.z = *reinterpret_cast<uint32_t*>(&t);
-    t = __floats2bfloat162_rn(v[6], v[7]); o.w = *reinterpret_cast<uint32_t*>(&t);
-    return o;
-}
-
-// Q and K: groups along d.  x [rows_total, d] with rows_total = B*H*N.  Thread t owns
-// elements [8t, 8t+8).  scale (optional) is [Hkv, d]; head h reads row map.kv_of[h].
-template <typename T>
-__global__ void __launch_bounds__(256)
-quantize_rows_kernel(const uint16_t* __restrict__ x, const float* __restrict__ scale, HeadMap map,
-                     int H, int N, int d, long long n_units, uint8_t* __restrict__ codes,
-                     uint32_t* __restrict__ meta, uint16_t* __restrict__ img,
-                     float* __restrict__ mu_out, float* __restrict__ ksum_out)
-{
-    long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= n_units) return;                        // n_units % 32 == 0: whole warps leave together
-    long long e0 = t * 8;
-    long long row = e0 / d;
-    int c0 = (int)(e0 - row * d);
-    uint4 raw = __ldg(reinterpret_cast<const uint4*>(x) + t);
-    const uint16_t* r16 = reinterpret_cast<const uint16_t*>(&raw);
-    float v[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = In16<T>::to_f(r16[i]);
-    if (scale) {
-        int h = (int)((row / N) % H);
-        const float4* sp = reinterpret_cast<const float4*>(scale + (long long)map.kv_of[h] * d + c0);
-        float4 s0 = __ldg(sp), s1 = __ldg(sp + 1);
-        const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
-#pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = In16<T>::round(v[i] * sv[i]);
-    }
-    if (mu_out || ksum_out) {
-        // Q-Mean auxiliary (Algorithm 1 lines 2 and 6).  A row of d channels sits in d/8 consecutive,
-        // aligned lanes; the sum runs in double, where it is exact for any row whose values span fewer
-        // than ~40 binades, so its order does not matter.
-        double sum = 0.0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) sum += (double)v[i];
-        for (int off = 1; off < d / 8; off <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-        if (mu_out) {                                // q_z = round_in(q~ - mu), mu = FP16(mean)
-            const float mu = __half2float(__double2half(sum / (double)d));
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = In16<T>::round_d((double)v[i] - (double)mu);
-            if (c0 == 0) mu_out[row] = mu;
-        } else if (c0 == 0) {
-            ksum_out[row] = __half2float(__double2half(sum));
-        }
-    }
-    float dq[8];
-    uint32_t mw;
-    uint32_t nib = quantize8(v, threadIdx.x & 7, dq, mw);
-    reinterpret_cast<uint32_t*>(codes)[t] = nib;
-    reinterpret_cast<uint4*>(img)[t] = pack_bf16x8(dq);
-    if ((threadIdx.x & 7) == 0) meta[t >> 3] = mw;
-}
-
-// V: groups of 64 tokens per channel; outputs are stored transposed ([.., d, N]).
-// One CTA transposes a 64-token x 64-channel tile through shared memory; 512 threads =
-// 64 channels x 8 lanes.
-template <typename T>
-__global__ void __launch_bounds__(512)
-quantize_tokens_kernel(const uint16_t* __restrict__ x, int N, int d, uint8_t* __restrict__ codes,
-                       uint32_t* __restrict__ meta, uint16_t* __restrict__ img)
-{
-    __shared__ uint16_t tile[64][72];                // +8 pad: 144-byte rows keep 16-byte alignment
-    const int tok0 = blockIdx.x * 64, ch0 = blockIdx.y * 64;
-    const long long bh = blockIdx.z;
-    const uint16_t* src = x + (bh * N + tok0) * (long long)d + ch0;
+// 16-bit input pairs <-> fp32, and the rounding of a smoothed pair back to the input dtype.
+template <typename T> struct Pair16;
+template <> struct Pair16<__nv_bfloat16> {
+    static __device__ __forceinline__ void unpack(uint32_t w, float& lo, float& hi)
     {
-        int r = threadIdx.x >> 3, c8 = threadIdx.x & 7;          // 64 rows x 8 chunks of 16 bytes
-        uint4 raw = __ldg(reinterpret_cast<const uint4*>(src + (long long)r * d) + c8);
-        *reinterpret_cast<uint4*>(&tile[r][c8 * 8]) = raw;
+        lo = __uint_as_float(w << 16);
+        hi = __uint_as_float(w & 0xFFFF0000u);
+    }
+    static __device__ __forceinline__ uint32_t round_pack(float lo, float hi)
+    {
+        uint32_t r;
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+        return r;
+    }
+};
+template <> struct Pair16<__half> {
+    static __device__ __forceinline__ void unpack(uint32_t w, float& lo, float& hi)
+    {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w));
+        lo = f.x;
+        hi = f.y;
+    }
+    static __device__ __forceinline__ uint32_t round_pack(float lo, float hi)
+    {
+        uint32_t r;
+        asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+        return r;
+    }
+};
+
+struct QuantJob {                     // one launch quantizes Q, K and V (any of them may be absent)
+    const uint16_t *q, *k, *v;        // [B,Hq,N,d], [B,Hkv,N,d], [B,Hkv,N,d]
+    const float *s, *inv_s;           // [Hkv,d] Smooth-QK factors for Q and K, or null
+    uint8_t *q_codes, *k_codes, *v_codes;
+    uint32_t *q_meta, *k_meta, *v_meta;
+    uint16_t *q_img, *k_img, *v_img;
+    float *q_mu, *k_sum;              // Q-Mean auxiliary outputs or null
+    int Hq, Hkv, N, d;
+    unsigned q_blocks, k_blocks;      // CTAs [0, q_blocks) take Q, the next k_blocks K, the rest V
+    unsigned row_blocks_per_head;     // N * d / 8 / ROW_UNITS_PER_CTA
+    HeadMap qmap;
+};
+
+constexpr int QUANT_THREADS = 256;
+constexpr int ROW_UNITS_PER_THREAD = 2;
+constexpr int ROW_UNITS_PER_CTA = QUANT_THREADS * ROW_UNITS_PER_THREAD;
+
+// Q and K: groups along d.  One head is N*d/8 units of 8 channels; a CTA takes 512 consecutive
+// units, thread t the units t and t + 256 (both loads are issued before any arithmetic).  The two
+// units share their channel offset, hence their Smooth-QK factors.
+template <typename T>
+__device__ __forceinline__ void quantize_rows_cta(const uint16_t* __restrict__ x, const float* __restrict__ scale,
+                                                  int kv_row, long long head, unsigned blk_in_head, int N, int d,
+                                                  uint8_t* __restrict__ codes, uint32_t* __restrict__ meta,
+                                                  uint16_t* __restrict__ img, float* __restrict__ mu_out,
+                                                  float* __restrict__ ksum_out)
+{
+    const int upr = d >> 3;                                                   // units per row
+    const unsigned u0 = blk_in_head * ROW_UNITS_PER_CTA + threadIdx.x;        // unit inside the head
+    const long long base = head * (long long)N * upr;                         // first unit of the head
+    const int c0 = (int)(u0 & (unsigned)(upr - 1)) << 3;
+    uint4 raw[ROW_UNITS_PER_THREAD];
+#pragma unroll
+    for (int r = 0; r < ROW_UNITS_PER_THREAD; ++r)
+        raw[r] = __ldg(reinterpret_cast<const uint4*>(x) + base + u0 + r * QUANT_THREADS);
+    float sv[8];
+    if (scale) {
+        const float4* sp = reinterpret_cast<const float4*>(scale + (long long)kv_row * d + c0);
+        const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1);
+        sv[0] = s0.x; sv[1] = s0.y; sv[2] = s0.z; sv[3] = s0.w;
+        sv[4] = s1.x; sv[5] = s1.y; sv[6] = s1.z; sv[7] = s1.w;
+    }
+#pragma unroll
+    for (int r = 0; r < ROW_UNITS_PER_THREAD; ++r) {
+        const unsigned u = u0 + r * QUANT_THREADS;
+        const long long t = base + u;
+        const uint32_t rw[4] = {raw[r].x, raw[r].y, raw[r].z, raw[r].w};
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) Pair16<T>::unpack(rw[i], v[2 * i], v[2 * i + 1]);
+        if (scale) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                Pair16<T>::unpack(Pair16<T>::round_pack(v[2 * i] * sv[2 * i], v[2 * i + 1] * sv[2 * i + 1]),
+                                  v[2 * i], v[2 * i + 1]);
+        }
+        if (mu_out || ksum_out) {
+            // Q-Mean auxiliary (Algorithm 1 lines 2 and 6).  A row of d channels sits in d/8 consecutive,
+            // aligned lanes; the sum runs in double, where it is exact for any row whose values span fewer
+            // than ~40 binades, so its order does not matter.
+            const long long row = head * N + (u >> (31 - __clz(upr)));
+            double sum = 0.0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sum += (double)v[i];
+            for (int off = 1; off < upr; off <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+            if (mu_out) {                                // q_z = round_in(q~ - mu), mu = FP16(mean)
+                const float mu = __half2float(__double2half(sum / (double)d));
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] = In16<T>::round_d((double)v[i] - (double)mu);
+                if (c0 == 0) mu_out[row] = mu;
+            } else if (c0 == 0) {
+                ksum_out[row] = __half2float(__double2half(sum));
+            }
+        }
+        uint32_t w[4], mw;
+        const uint32_t nib = quantize8(v, threadIdx.x & 7, w, mw);
+        reinterpret_cast<uint32_t*>(codes)[t] = nib;
+        reinterpret_cast<uint4*>(img)[t] = make_uint4(w[0], w[1], w[2], w[3]);
+        if ((threadIdx.x & 7) == 0) meta[t >> 3] = mw;
+    }
+}
+
+// V: groups of 64 tokens per channel; outputs are stored transposed ([.., d, N]).  One CTA
+// transposes a 64-token x 64-channel tile through shared memory.  The tile is kept as 64 rows of
+// 8 16-byte chunks, chunk c of row r stored at position c ^ (r >> 3), so that both the row-wise
+// 16-byte stores and the column-wise 4-byte reads (a thread reads two adjacent channels of 8
+// consecutive tokens) are free of bank conflicts.  256 threads = 32 channel pairs x 8 lanes.
+template <typename T>
+__device__ __forceinline__ void quantize_tokens_cta(const uint16_t* __restrict__ x, long long bh, int tok0, int ch0,
+                                                    int N, int d, uint8_t* __restrict__ codes,
+                                                    uint32_t* __restrict__ meta, uint16_t* __restrict__ img)
+{
+    __shared__ uint4 tile[64 * 8];
+    const uint16_t* src = x + (bh * N + tok0) * (long long)d + ch0;
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+        const int idx = threadIdx.x + it * QUANT_THREADS;
+        const int r = idx >> 3, c8 = idx & 7;
+        tile[r * 8 + (c8 ^ (r >> 3))] = __ldg(reinterpret_cast<const uint4*>(src + (long long)r * d) + c8);
     }
     __syncthreads();
-    const int c = threadIdx.x >> 3, j = threadIdx.x & 7;          // channel, level-2 unit
-    float v[8];
+    const int cp = threadIdx.x >> 3, j = threadIdx.x & 7;          // channel pair, level-2 unit
+    const uint32_t* tw = reinterpret_cast<const uint32_t*>(tile);
+    float va[8], vb[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = In16<T>::to_f(tile[8 * j + i][c]);
-    float dq[8];
-    uint32_t mw;
-    uint32_t nib = quantize8(v, j, dq, mw);
-    const long long orow = bh * d + ch0 + c;                      // row of the transposed outputs
-    reinterpret_cast<uint32_t*>(codes + orow * (N / 2) + tok0 / 2)[j] = nib;
-    reinterpret_cast<uint4*>(img + orow * (long long)N + tok0)[j] = pack_bf16x8(dq);
-    if (j == 0) meta[orow * (N / 64) + tok0 / 64] = mw;
+    for (int i = 0; i < 8; ++i)
+        Pair16<T>::unpack(tw[(8 * j + i) * 32 + ((((cp >> 2) ^ j) << 2) | (cp & 3))], va[i], vb[i]);
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+        uint32_t w[4], mw;
+        const uint32_t nib = quantize8(c ? vb : va, j, w, mw);
+        const long long orow = bh * d + ch0 + 2 * cp + c;             // row of the transposed outputs
+        reinterpret_cast<uint32_t*>(codes + orow * (N / 2) + tok0 / 2)[j] = nib;
+        reinterpret_cast<uint4*>(img + orow * (long long)N + tok0)[j] = make_uint4(w[0], w[1], w[2], w[3]);
+        if (j == 0) meta[orow * (N / 64) + tok0 / 64] = mw;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(QUANT_THREADS)
+quantize_qkv_kernel(const __grid_constant__ QuantJob job)
+{
+    unsigned blk = blockIdx.x;
+    if (blk < job.q_blocks + job.k_blocks) {
+        const bool is_q = blk < job.q_blocks;
+        if (!is_q) blk -= job.q_blocks;
+        const unsigned head = blk / job.row_blocks_per_head;             // b * H + h
+        const unsigned in_head = blk - head * job.row_blocks_per_head;
+        if (is_q)
+            quantize_rows_cta<T>(job.q, job.s, job.qmap.kv_of[head % (unsigned)job.Hq], head, in_head, job.N, job.d,
+                                 job.q_codes, job.q_meta, job.q_img, job.q_mu, nullptr);
+        else
+            quantize_rows_cta<T>(job.k, job.inv_s, (int)(head % (unsigned)job.Hkv), head, in_head, job.N, job.d,
+                                 job.k_codes, job.k_meta, job.k_img, nullptr, job.k_sum);
+    } else {
+        blk -= job.q_blocks + job.k_blocks;
+        const unsigned tok_blocks = job.N / 64, ch_blocks = job.d / 64;
+        const unsigned tb = blk % tok_blocks, rest = blk / tok_blocks;
+        const unsigned cb = rest % ch_blocks, bh = rest / ch_blocks;
+        quantize_tokens_cta<T>(job.v, bh, tb * 64, cb * 64, job.N, job.d, job.v_codes, job.v_meta, job.v_img);
+    }
 }
 
 // Calibration: per (sample, kv head, channel) maximum magnitude over tokens (and over the query
@@ -199,36 +304,30 @@ __global__ void smooth_finalize_kernel(const float* __restrict__ kmax, const flo
 }
 
 // ------------------------------------------------------------------------------- launchers
-template <typename T>
-static cudaError_t launch_rows(const void* x, const float* scale, const HeadMap& map, int B, int H,
-                               int N, int d, uint8_t* codes, uint32_t* meta, void* img, float* mu_out,
-                               float* ksum_out, cudaStream_t st)
+cudaError_t launch_quantize_qkv(int dtype, const hifa4_shape& sh, const HeadMap& qmap, const void* q,
+                                const void* k, const void* v, const float* s, const float* inv_s,
+                                const hifa4_qkv& out, cudaStream_t st)
 {
-    long long units = (long long)B * H * N * d / 8;
-    unsigned blocks = (unsigned)((units + 255) / 256);
-    quantize_rows_kernel<T><<<blocks, 256, 0, st>>>((const uint16_t*)x, scale, map, H, N, d, units,
-                                                    codes, meta, (uint16_t*)img, mu_out, ksum_out);
-    count_launch();
-    return cudaGetLastError();
-}
-
-cudaError_t launch_quantize_rows(int dtype, const void* x, const float* scale, const HeadMap& map,
-                                 int B, int H, int N, int d, uint8_t* codes, uint32_t* meta,
-                                 void* img, float* mu_out, float* ksum_out, cudaStream_t st)
-{
-    return dtype == HIFA4_F16
-               ? launch_rows<__half>(x, scale, map, B, H, N, d, codes, meta, img, mu_out, ksum_out, st)
-               : launch_rows<__nv_bfloat16>(x, scale, map, B, H, N, d, codes, meta, img, mu_out, ksum_out, st);
-}
-
-cudaError_t launch_quantize_tokens(int dtype, const void* x, int B, int H, int N, int d,
-                                   uint8_t* codes, uint32_t* meta, void* img, cudaStream_t st)
-{
-    dim3 grid(N / 64, d / 64, B * H);
+    QuantJob job{};
+    job.q = (const uint16_t*)q; job.k = (const uint16_t*)k; job.v = (const uint16_t*)v;
+    job.s = s; job.inv_s = inv_s;
+    job.q_codes = out.q_codes; job.k_codes = out.k_codes; job.v_codes = out.v_codes;
+    job.q_meta = out.q_meta; job.k_meta = out.k_meta; job.v_meta = out.v_meta;
+    job.q_img = (uint16_t*)out.q_mma; job.k_img = (uint16_t*)out.k_mma; job.v_img = (uint16_t*)out.v_mma;
+    job.q_mu = out.q_mu; job.k_sum = out.k_sum;
+    job.Hq = sh.Hq; job.Hkv = sh.Hkv; job.N = sh.N; job.d = sh.d;
+    job.row_blocks_per_head = (unsigned)((long long)sh.N * sh.d / 8 / ROW_UNITS_PER_CTA);
+    job.q_blocks = q ? (unsigned)sh.B * sh.Hq * job.row_blocks_per_head : 0u;
+    job.k_blocks = k ? (unsigned)sh.B * sh.Hkv * job.row_blocks_per_head : 0u;
+    const unsigned v_blocks = v ? (unsigned)sh.B * sh.Hkv * (sh.N / 64) * (sh.d / 64) : 0u;
+    job.qmap = qmap;
+    const unsigned long long total = (unsigned long long)job.q_blocks + job.k_blocks + v_blocks;
+    if (total == 0) return cudaSuccess;
+    if (total > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
     if (dtype == HIFA4_F16)
-        quantize_tokens_kernel<__half><<<grid, 512, 0, st>>>((const uint16_t*)x, N, d, codes, meta, (uint16_t*)img);
+        quantize_qkv_kernel<__half><<<(unsigned)total, QUANT_THREADS, 0, st>>>(job);
     else
-        quantize_tokens_kernel<__nv_bfloat16><<<grid, 512, 0, st>>>((const uint16_t*)x, N, d, codes, meta, (uint16_t*)img);
+        quantize_qkv_kernel<__nv_bfloat16><<<(unsigned)total, QUANT_THREADS, 0, st>>>(job);
     count_launch();
     return cudaGetLastError();
 }
