@@ -20,9 +20,12 @@
 
 namespace hifa4 {
 
+#ifndef HIFA4_WS64_KS128
+#define HIFA4_WS64_KS128 2
+#endif
 template <int D_>
 struct WS64 {
-    static constexpr int D = D_, BC = 64, STAGES = 2, KS = 2;
+    static constexpr int D = D_, BC = 64, STAGES = 2, KS = (D_ == 128) ? HIFA4_WS64_KS128 : 2;
     static constexpr int NSW = 4 * KS, THREADS = (NSW + 2) * 32, W_TMA = NSW, W_MMA = NSW + 1;
     static constexpr int KPT = BC / KS, NU = KPT / 8;       // 32 keys = 4 level-2 units per thread and tile
     static constexpr int QSUB = D / 64;                     // 64-channel sub-tiles of Q and K
@@ -35,7 +38,7 @@ struct WS64 {
     static constexpr int V_OFF = K_OFF + STAGES * K_STAGE;
     static constexpr int MISC_OFF = V_OFF + STAGES * V_STAGE;
     static constexpr int XCHG_OFF = MISC_OFF + 256;         // partial row maxima [2 parities][2 splits][128 rows]
-    static constexpr int SMEM_BYTES = XCHG_OFF + 2 * 2 * 128 * 4 + 1024;
+    static constexpr int SMEM_BYTES = XCHG_OFF + 2 * KS * 128 * 4 + 1024;
     static constexpr int O_COLS = D + 16;
     static constexpr bool Q_IN_TMEM = (D == 256);
     static constexpr int QT_COL = 272;                      // d = 256 only
@@ -221,6 +224,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         // channels of its row = 64 columns of packed BF16 pairs.  (d = 128: the issuer waits for the
         // Q load itself.)
         if constexpr (C::Q_IN_TMEM) {
+            static_assert(!C::Q_IN_TMEM || KS == 2, "the Q copy splits a row over two threads");
             if (wait64(bar(BAR_Q), 0, abort_flag)) {
                 const int sw = r_loc & 7;
 #pragma unroll
@@ -250,11 +254,12 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             tc_fence_after();
             float p[KPT];
             {
-                uint32_t r[32];
-                tmem_ld32(t_lane + S_COL + kq * KPT, r);
+                uint32_t r[KPT];
+                if constexpr (KPT == 32) tmem_ld32(t_lane + S_COL + kq * KPT, r);
+                else tmem_ld16(t_lane + S_COL + kq * KPT, r);
                 tmem_wait_ld();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) p[i] = __uint_as_float(r[i]);
+                for (int i = 0; i < KPT; ++i) p[i] = __uint_as_float(r[i]);
             }
             tc_fence_before();                                 // S(jt) is in registers: S(jt+1) may overwrite it
             __syncwarp();
@@ -288,11 +293,13 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                     for (int i = 0; i < w; ++i) t4[i] = fmaxf(t4[i], t4[i + w]);
                 mx = t4[0];
             }
-            xmax[(par * 2 + kq) * 128 + r_loc] = mx;
+            xmax[(par * KS + kq) * 128 + r_loc] = mx;
             __syncwarp();
             if (lane == 0) mbar_arrive(xbar);
             if (!wait64(xbar, par, abort_flag)) { fail(9); ok = false; break; }
-            mx = fmaxf(mx, xmax[(par * 2 + (kq ^ 1)) * 128 + r_loc]);   // the tile is one 64-key group: row max = group max
+#pragma unroll
+            for (int o = 1; o < KS; ++o)                       // the tile is one 64-key group: row max = group max
+                mx = fmaxf(mx, xmax[(par * KS + (kq ^ o)) * 128 + r_loc]);
 
             const float m_new = fmaxf(m_run, f16_round(mx * args.c0));
             float rsc = 1.f;
@@ -318,8 +325,44 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 if (!wait64(bar(BAR_PV), par ^ 1u, abort_flag)) { fail(10); ok = false; break; }
                 tc_fence_after();
             }
-            tmem_st16(t_lane + P_COL + kq * (KPT / 2), w);
+            if constexpr (NU == 4) tmem_st16(t_lane + P_COL + kq * (KPT / 2), w);
+            else tmem_st8(t_lane + P_COL + kq * (KPT / 2), w);
             // rescale history (line 8): each half of the row's threads owns half of the d + 16 columns
+            if constexpr (D == 128 && KS == 2) {            // all of the thread's 72 columns in one round trip
+                if (__any_sync(0xffffffffu, rsc != 1.f)) {
+                    const uint32_t t_o = t_lane + kq * 72;
+                    const uint64_t rr = pack2(rsc, rsc);
+                    uint32_t r0[32], r1[32], r2[4], r3[4];
+                    tmem_ld32(t_o, r0);
+                    tmem_ld32(t_o + 32, r1);
+                    tmem_ld4(t_o + 64, r2);
+                    tmem_ld4(t_o + 68, r3);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float x0, x1;
+                        unpack2(mul2(pack2(__uint_as_float(r0[i]), __uint_as_float(r0[i + 1])), rr), x0, x1);
+                        r0[i] = __float_as_uint(x0);
+                        r0[i + 1] = __float_as_uint(x1);
+                    }
+                    tmem_st32(t_o, r0);
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float x0, x1;
+                        unpack2(mul2(pack2(__uint_as_float(r1[i]), __uint_as_float(r1[i + 1])), rr), x0, x1);
+                        r1[i] = __float_as_uint(x0);
+                        r1[i + 1] = __float_as_uint(x1);
+                    }
+                    tmem_st32(t_o + 32, r1);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        r2[i] = __float_as_uint(__uint_as_float(r2[i]) * rsc);
+                        r3[i] = __float_as_uint(__uint_as_float(r3[i]) * rsc);
+                    }
+                    tmem_st4(t_o + 64, r2);
+                    tmem_st4(t_o + 68, r3);
+                }
+            } else
             if (__any_sync(0xffffffffu, rsc != 1.f)) {
                 constexpr int CW = O_COLS / KS;                // 136 or 72
                 const uint32_t t_o = t_lane + kq * CW;
@@ -366,11 +409,11 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 if (args.dbg.l_out) args.dbg.l_out[dbg_slot * 128 + r_loc] = ell;
                 if (args.dbg.m_out) args.dbg.m_out[dbg_slot * 128 + r_loc] = m_run;
             }
-            const size_t orow = ((size_t)bh_q * N + row) * D + kq * (D / 2);
+            const size_t orow = ((size_t)bh_q * N + row) * D + kq * (D / KS);
 #pragma unroll
-            for (int cc = 0; cc < D / 64; ++cc) {
+            for (int cc = 0; cc < D / KS / 32; ++cc) {
                 uint32_t r[32];
-                tmem_ld32(t_lane + kq * (D / 2) + cc * 32, r);
+                tmem_ld32(t_lane + kq * (D / KS) + cc * 32, r);
                 tmem_wait_ld();
                 if (row < N) {
                     float o[32];
