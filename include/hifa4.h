@@ -101,7 +101,11 @@ typedef struct { float rho_K, T_KQ; int branch; float alpha; } hifa4_calib_stats
  *               of the result: P is quantized under the running maximum that
  *               holds after each Bc keys (Algorithm 1 lines 7-10).
  *   normalizer  0: consistent (P-Reordering, normalizer = rowsum of P-hat via
- *               the ones column); 1 (mismatched) is not built.
+ *               the ones column); 1: mismatched, the normalizer is accumulated
+ *               from the unquantized FP16 P while PV consumes P-hat (the
+ *               "Direct" baseline of "P-Reordering"; Theorem 1's O_mis).  Mode 1
+ *               is an ablation: it runs on a one-thread-per-row kernel, several
+ *               times slower than mode 0.
  *   qmean       1: add the Q-Mean correction mu_i * k_sum_j to the raw scores (line 6; scaled by the
  *               softmax scale together with them); needs qkv->q_mu and qkv->k_sum filled by
  *               hifa4_quantize_qkv.  0: no correction (the Q buffers must then hold un-centred Q).
@@ -130,6 +134,18 @@ typedef struct {
     float* l_out;
     float* m_out;
 } hifa4_debug;
+
+/* Histogram of the per-tile mass error of P-hat ("P-Reordering", Theorem 1 and the
+ * figure of its empirical validation): for every query row and every Bc-key tile whose
+ * P is not all zero, eps = sum_j P-hat_j / sum_j P_j - 1 over the keys of the tile, both
+ * sums exact.  hist: device array of n_bins + 2 counters that the call ADDS to (clear it
+ * first): bin k counts lo + k*w <= eps < lo + (k+1)*w with w = (hi - lo)/n_bins; entry
+ * n_bins counts eps < lo, entry n_bins + 1 counts eps >= hi. */
+typedef struct {
+    unsigned long long* hist;
+    int n_bins;
+    double lo, hi;
+} hifa4_mass_stats;
 
 const char* hifa4_status_string(int status);
 
@@ -205,6 +221,14 @@ size_t hifa4_attention_workspace_bytes(const hifa4_shape* shape, const hifa4_att
 int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv,
                         const hifa4_attn_params* prm, void* out, void* workspace,
                         const hifa4_debug* dbg, int* d_status, void* stream);
+
+/* hifa4_attention_fwd that also fills the mass-error histogram of P-hat (see
+ * hifa4_mass_stats; "P-Reordering", Theorem 1).  Same arguments and result as
+ * hifa4_attention_fwd (either normalizer mode); stats must be non-NULL with
+ * n_bins >= 1 and lo < hi.  Analysis path: it runs on the one-thread-per-row kernel. */
+int hifa4_attention_fwd_stats(const hifa4_shape* shape, const hifa4_qkv* qkv,
+                              const hifa4_attn_params* prm, void* out, void* workspace,
+                              const hifa4_mass_stats* stats, int* d_status, void* stream);
 
 /* Workspace for hifa4_attention_fwd_raw: all hifa4_qkv buffers (each rounded up
  * to 256 bytes; the two Q-Mean vectors only when prm->qmean = 1) plus the

@@ -54,6 +54,10 @@ class _CalibStats(C.Structure):
     _fields_ = [("rho_K", C.c_float), ("T_KQ", C.c_float), ("branch", C.c_int), ("alpha", C.c_float)]
 
 
+class _MassStats(C.Structure):
+    _fields_ = [("hist", C.c_void_p), ("n_bins", C.c_int), ("lo", C.c_double), ("hi", C.c_double)]
+
+
 _lib = None
 
 
@@ -95,6 +99,10 @@ def lib():
         L.hifa4_attention_fwd.restype = C.c_int
         L.hifa4_attention_fwd.argtypes = [C.POINTER(_Shape), C.POINTER(_QKV), C.POINTER(_AttnParams),
                                           C.c_void_p, C.c_void_p, C.POINTER(_Debug), C.c_void_p, C.c_void_p]
+        L.hifa4_attention_fwd_stats.restype = C.c_int
+        L.hifa4_attention_fwd_stats.argtypes = [C.POINTER(_Shape), C.POINTER(_QKV), C.POINTER(_AttnParams),
+                                                C.c_void_p, C.c_void_p, C.POINTER(_MassStats), C.c_void_p,
+                                                C.c_void_p]
         L.hifa4_attention_fwd_raw.restype = C.c_int
         L.hifa4_attention_fwd_raw.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.c_void_p,
                                               C.c_void_p, C.c_void_p, C.POINTER(_AttnParams), C.c_void_p,
@@ -108,7 +116,7 @@ STATIC_CALIB_MAX_FLOATS = 1 << 20
 EXPORTS = ("hifa4_status_string", "hifa4_get_counters", "hifa4_smooth_calibrate",
            "hifa4_smooth_calibrate_static", "hifa4_quant_bytes",
            "hifa4_quantize_qkv", "hifa4_attention_workspace_bytes", "hifa4_attention_fwd",
-           "hifa4_attention_raw_workspace_bytes", "hifa4_attention_fwd_raw")
+           "hifa4_attention_fwd_stats", "hifa4_attention_raw_workspace_bytes", "hifa4_attention_fwd_raw")
 
 
 def status_string(status: int) -> str:
@@ -266,12 +274,13 @@ def quantize_qkv(q, k, v, s=None, inv_s=None, q_to_kv=None, out: QuantizedQKV | 
 
 
 def attention_fwd(qkv: QuantizedQKV, causal: bool, Bc: int = 128, out_dtype=F32, out=None,
-                  debug_blocks=None, d_status=None, softmax_scale=0.0, Br=128, qmean=False):
+                  debug_blocks=None, d_status=None, softmax_scale=0.0, Br=128, qmean=False, normalizer=0):
     """Fused attention forward on quantized operands.  Returns out [B,Hq,N,d], or
     (out, dict(p_codes, p_step, l, m)) when debug_blocks (a list of (b, h, query block)) is given."""
     dev = qkv.q_mma.device
     sh = _shape(qkv.B, qkv.Hq, qkv.Hkv, qkv.N, qkv.d, qkv.in_dtype, qkv.q_to_kv)
-    prm = _params(causal, Bc, out_dtype, Br=Br, softmax_scale=softmax_scale, qmean=int(qmean))
+    prm = _params(causal, Bc, out_dtype, Br=Br, softmax_scale=softmax_scale, qmean=int(qmean),
+                  normalizer=int(normalizer))
     if out is None:
         out = torch.empty((qkv.B, qkv.Hq, qkv.N, qkv.d), dtype=_TORCH_DT[out_dtype], device=dev)
     st = qkv.struct()
@@ -292,6 +301,24 @@ def attention_fwd(qkv: QuantizedQKV, causal: bool, Bc: int = 128, out_dtype=F32,
                                    _ptr(d_status), _stream())
     _check(rc, "hifa4_attention_fwd")
     return (out, dump) if debug_blocks else out
+
+
+def attention_fwd_stats(qkv: QuantizedQKV, causal: bool, n_bins: int, lo: float, hi: float, Bc: int = 128,
+                        out_dtype=F32, hist=None, d_status=None, softmax_scale=0.0, qmean=False, normalizer=0):
+    """Attention forward that also adds to the histogram of the per-(row, key tile) mass error of P-hat.
+    Returns (out, hist) with hist a device int64 tensor of n_bins + 2 counters (last two: below lo, at or above hi)."""
+    dev = qkv.q_mma.device
+    sh = _shape(qkv.B, qkv.Hq, qkv.Hkv, qkv.N, qkv.d, qkv.in_dtype, qkv.q_to_kv)
+    prm = _params(causal, Bc, out_dtype, softmax_scale=softmax_scale, qmean=int(qmean), normalizer=int(normalizer))
+    out = torch.empty((qkv.B, qkv.Hq, qkv.N, qkv.d), dtype=_TORCH_DT[out_dtype], device=dev)
+    if hist is None:
+        hist = torch.zeros(n_bins + 2, dtype=torch.int64, device=dev)
+    st = qkv.struct()
+    stats = _MassStats(hist.data_ptr(), int(n_bins), float(lo), float(hi))
+    rc = lib().hifa4_attention_fwd_stats(C.byref(sh), C.byref(st), C.byref(prm), _ptr(out), None,
+                                         C.byref(stats), _ptr(d_status), _stream())
+    _check(rc, "hifa4_attention_fwd_stats")
+    return out, hist
 
 
 def attention_raw_workspace_bytes(B, Hq, Hkv, N, d, in_dtype, causal, Bc, out_dtype=F32, qmean=False) -> int:

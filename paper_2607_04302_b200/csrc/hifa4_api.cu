@@ -160,7 +160,8 @@ static int check_attn(const hifa4_shape* shape, const hifa4_attn_params* prm)
     if (prm->Bc != 64 && prm->Bc != 128) return HIFA4_ERR_UNSUPPORTED;
     if (shape->d == 256 && prm->Bc != 64) return HIFA4_ERR_UNSUPPORTED;
     if (prm->qmean != 0 && prm->qmean != 1) return HIFA4_ERR_INVALID_ARG;
-    if (prm->normalizer != 0 || prm->p_dtype != HIFA4_F16) return HIFA4_ERR_UNSUPPORTED;
+    if (prm->normalizer != 0 && prm->normalizer != 1) return HIFA4_ERR_INVALID_ARG;
+    if (prm->p_dtype != HIFA4_F16) return HIFA4_ERR_UNSUPPORTED;
     return HIFA4_OK;
 }
 
@@ -170,11 +171,10 @@ size_t hifa4_attention_workspace_bytes(const hifa4_shape* shape, const hifa4_att
     return 0;
 }
 
-int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
-                        void* out, void* workspace, const hifa4_debug* dbg, int* d_status,
-                        void* stream)
+static int attention_common(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
+                            void* out, const hifa4_debug* dbg, const hifa4_mass_stats* stats, int* d_status,
+                            void* stream)
 {
-    (void)workspace;
     g_calls[2].fetch_add(1, std::memory_order_relaxed);
     int rc = check_attn(shape, prm);
     if (rc) return rc;
@@ -193,7 +193,24 @@ int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv, const hi
     HeadMap qmap, kmap;
     if ((rc = build_map(shape->Hq, shape->Hkv, shape->q_to_kv, qmap, kmap))) return rc;
     if ((rc = check_arch())) return rc;
-    return launch_attention(*shape, qmap, *qkv, *prm, out, dbg, d_status, (cudaStream_t)stream);
+    return launch_attention(*shape, qmap, *qkv, *prm, out, dbg, stats, d_status, (cudaStream_t)stream);
+}
+
+int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
+                        void* out, void* workspace, const hifa4_debug* dbg, int* d_status,
+                        void* stream)
+{
+    (void)workspace;
+    return attention_common(shape, qkv, prm, out, dbg, nullptr, d_status, stream);
+}
+
+int hifa4_attention_fwd_stats(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
+                              void* out, void* workspace, const hifa4_mass_stats* stats, int* d_status,
+                              void* stream)
+{
+    (void)workspace;
+    if (!stats || !stats->hist || stats->n_bins < 1 || !(stats->lo < stats->hi)) return HIFA4_ERR_INVALID_ARG;
+    return attention_common(shape, qkv, prm, out, nullptr, stats, d_status, stream);
 }
 
 static size_t qkv_layout(const hifa4_shape* shape, int qmean, char* base, hifa4_qkv* o)

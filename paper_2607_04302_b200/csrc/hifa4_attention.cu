@@ -11,7 +11,9 @@
 
 namespace hifa4 {
 
-template <int D, int BC>
+// AUX: the variant that also keeps the row sums of the unquantized P (exactly, in 2^-24 fixed point:
+// P is an FP16 value), for the mismatched normalizer and for the mass-error histogram.
+template <int D, int BC, bool AUX>
 __global__ void __launch_bounds__(128, 1)
 attention_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                      const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnArgs args)
@@ -79,6 +81,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
         const int last_key = args.causal ? min(q0 + 127, N - 1) : N - 1;
         const int n_tiles = last_key / BC + 1;
         float m_run = -INFINITY;                          // FP16 value held in a float
+        float ell_p = 0.f;                                // AUX: normalizer accumulated from P (mismatched)
         const float LOG2E = 1.4426950408889634f;
         // Q-Mean correction (line 6): mu of this row, channel sum of every key of the KV head
         const float mu_row = (args.qmean && row < N) ? args.q_mu[(size_t)bh_q * N + row] : 0.f;
@@ -139,6 +142,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
             if (jt > 0) {
                 float rsc = 1.f;
                 if (m_new != m_run) rsc = f16_round(ex2_approx((m_run - m_new) * LOG2E));
+                if (AUX) ell_p *= rsc;
                 if (__any_sync(0xffffffffu, rsc != 1.f)) {
 #pragma unroll
                     for (int cc = 0; cc < C::O_COLS / 16; ++cc) {
@@ -156,6 +160,8 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
             const float mL = m_run * LOG2E;
 
             // ---- P = exp(S - m) in FP16 (line 9), P-hat = HIF4(P) per 64 keys (line 10)
+            uint32_t p_fix = 0;                           // AUX: sum of P over the tile in units of 2^-24 (< 2^32)
+            double ph_sum = 0.0;                          // AUX: sum of P-hat over the tile (exact)
 #pragma unroll
             for (int gq = 0; gq < C::PSUB; ++gq) {
                 float p[64];
@@ -181,7 +187,23 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
                     if (args.dbg.p_codes) dc = args.dbg.p_codes + r_idx * N + j0 + gq * 64;
                     if (args.dbg.p_step) ds = args.dbg.p_step + r_idx * (N / 4) + (j0 + gq * 64) / 4;
                 }
-                quantize_p64(p, p_s + gq * C::P_SUB_BYTES, tid, dc, ds);
+                float gsum;
+                quantize_p64(p, p_s + gq * C::P_SUB_BYTES, tid, dc, ds, AUX ? &gsum : nullptr);
+                if (AUX) {
+                    ph_sum += (double)gsum;
+#pragma unroll
+                    for (int i = 0; i < 64; ++i) p_fix += __float2uint_rz(p[i] * 16777216.f);
+                }
+            }
+            if (AUX) {
+                const double p_sum = (double)p_fix * (1.0 / 16777216.0);
+                ell_p = __double2float_rn((double)ell_p + p_sum);     // one rounding per tile, as for the MMA's l
+                if (args.hist && row < N && p_fix != 0) {             // per (row, key tile) mass error of P-hat
+                    const double eps = ph_sum / p_sum - 1.0;
+                    const double x = floor((eps - args.hist_lo) * args.hist_inv_w);
+                    const int bin = x < 0.0 ? args.n_bins : (x >= (double)args.n_bins ? args.n_bins + 1 : (int)x);
+                    atomicAdd(args.hist + bin, 1ull);
+                }
             }
             fence_proxy_async_smem();                     // P-hat tile -> visible to the MMA's smem reads
             tc_fence_before();
@@ -214,7 +236,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
             uint32_t lr[16];
             tmem_ld16(t_o + D, lr);
             tmem_wait_ld();
-            const float ell = __uint_as_float(lr[0]);
+            const float ell = (AUX && args.normalizer) ? ell_p : __uint_as_float(lr[0]);
             const float l16 = f16_round(ell);
             if (dbg_slot >= 0 && row < N) {
                 if (args.dbg.l_out) args.dbg.l_out[dbg_slot * 128 + tid] = ell;
@@ -299,7 +321,7 @@ bool make_bf16_map(CUtensorMap* m, void* base, uint64_t heads, uint64_t rows, ui
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int D, int BC>
+template <int D, int BC, bool AUX>
 static int launch_cfg(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
     using C = Cfg<D, BC>;
@@ -307,7 +329,7 @@ static int launch_cfg(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArg
     if (!make_bf16_map(&mq, qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, D, 128)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, D, BC)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, D, sh.N, D)) return HIFA4_ERR_CUDA;
-    auto kern = attention_fwd_kernel<D, BC>;
+    auto kern = attention_fwd_kernel<D, BC, AUX>;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
@@ -321,8 +343,8 @@ static int launch_cfg(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArg
 }
 
 int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv& qkv,
-                     const hifa4_attn_params& prm, void* out, const hifa4_debug* dbg, int* d_status,
-                     cudaStream_t st)
+                     const hifa4_attn_params& prm, void* out, const hifa4_debug* dbg,
+                     const hifa4_mass_stats* stats, int* d_status, cudaStream_t st)
 {
     AttnArgs a;
     memset(&a, 0, sizeof(a));
@@ -344,8 +366,23 @@ int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv&
         a.dbg.p_codes = dbg->p_codes; a.dbg.p_step = dbg->p_step;
         a.dbg.l_out = dbg->l_out; a.dbg.m_out = dbg->m_out;
     }
-    if (sh.d == 64 && prm.Bc == 64) return launch_cfg<64, 64>(sh, qkv, a, st);
-    if (sh.d == 64 && prm.Bc == 128) return launch_cfg<64, 128>(sh, qkv, a, st);
+    a.normalizer = prm.normalizer ? 1 : 0;
+    if (stats) {
+        a.hist = stats->hist;
+        a.n_bins = stats->n_bins;
+        a.hist_lo = stats->lo;
+        a.hist_inv_w = (double)stats->n_bins / (stats->hi - stats->lo);
+    }
+    if (a.normalizer || a.hist) {                 // the one-thread-per-row kernel keeps the sums of P
+        if (sh.d == 64 && prm.Bc == 64) return launch_cfg<64, 64, true>(sh, qkv, a, st);
+        if (sh.d == 64 && prm.Bc == 128) return launch_cfg<64, 128, true>(sh, qkv, a, st);
+        if (sh.d == 128 && prm.Bc == 64) return launch_cfg<128, 64, true>(sh, qkv, a, st);
+        if (sh.d == 128 && prm.Bc == 128) return launch_cfg<128, 128, true>(sh, qkv, a, st);
+        if (sh.d == 256 && prm.Bc == 64) return launch_cfg<256, 64, true>(sh, qkv, a, st);
+        return HIFA4_ERR_UNSUPPORTED;
+    }
+    if (sh.d == 64 && prm.Bc == 64) return launch_cfg<64, 64, false>(sh, qkv, a, st);
+    if (sh.d == 64 && prm.Bc == 128) return launch_cfg<64, 128, false>(sh, qkv, a, st);
     if (sh.d == 128 && prm.Bc == 64) return launch_attention_ws64(sh, qkv, a, st);
     if (sh.d == 128 && prm.Bc == 128) return launch_attention_ws(sh, qkv, a, st);
     if (sh.d == 256 && prm.Bc == 64) return launch_attention_ws64(sh, qkv, a, st);

@@ -24,6 +24,10 @@ struct AttnArgs {
     int B, Hq, Hkv, N;
     int causal, out_dtype;
     float c0, c1;                 // sigma, sigma * log2(e)
+    int normalizer;               // 1: l accumulates the unquantized P (mismatched), not P-hat
+    unsigned long long* hist;     // mass-error histogram [n_bins + 2] or null
+    int n_bins;
+    double hist_lo, hist_inv_w;   // bin = floor((eps - lo) * inv_w)
     int qmean;                    // add mu_i * k_sum_j to the raw scores (Algorithm 1 line 6)
     const float* q_mu;            // [B,Hq,N]
     const float* k_sum;           // [B,Hkv,N]
@@ -83,8 +87,10 @@ __device__ __forceinline__ void exp2_f16_pair(float t0, float t1, float& e0, flo
 // max(need) = 2 or min(need) >= 1" is a = (n0 + n1 + 2) >> 2 and the shifts are max(n, a).
 template <int NU>
 __device__ __forceinline__ void quantize_p_units(const float (&p)[NU * 8], const float (&At)[NU * 2], float A,
-                                                 uint32_t (&w)[NU * 4], uint8_t* dump_codes, float* dump_step)
+                                                 uint32_t (&w)[NU * 4], uint8_t* dump_codes, float* dump_step,
+                                                 float* sum_out = nullptr)
 {
+    if (sum_out) *sum_out = 0.f;
     if (A == 0.f) {
 #pragma unroll
         for (int i = 0; i < NU * 4; ++i) w[i] = 0u;
@@ -121,6 +127,7 @@ __device__ __forceinline__ void quantize_p_units(const float (&p)[NU * 8], const
             for (int i = 0; i < 4; ++i) {
                 const float y = __fadd_rn(__fmul_rz(p[8 * u + 4 * h + i], inv_step), MAGIC);
                 v[i] = fmaf(y, step, negc);
+                if (sum_out) *sum_out += v[i];            // exact: every term is a multiple of S/4, the sum < 2^11 of them
                 if (dump_codes) packed |= (__float_as_uint(y) & 15u) << (8 * i);
             }
             asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h]) : "f"(v[1]), "f"(v[0]));
@@ -241,7 +248,7 @@ __device__ __forceinline__ void exp_quantize_units(const float (&acc)[NU * 8], c
 // Whole 64-key group held by one thread; the image goes to row `row` of a 128-byte-swizzled
 // shared-memory tile (the layout a K-major tcgen05 operand descriptor with SWIZZLE_128B reads).
 __device__ __forceinline__ void quantize_p64(const float (&p)[64], uint32_t p_sub_base, int row,
-                                             uint8_t* dump_codes, float* dump_step)
+                                             uint8_t* dump_codes, float* dump_step, float* sum_out = nullptr)
 {
     float At[16];
 #pragma unroll
@@ -251,7 +258,7 @@ __device__ __forceinline__ void quantize_p64(const float (&p)[64], uint32_t p_su
     for (int t = 0; t < 4; ++t) A4[t] = fmaxf(max3(At[4 * t], At[4 * t + 1], At[4 * t + 2]), At[4 * t + 3]);
     const float A = fmaxf(max3(A4[0], A4[1], A4[2]), A4[3]);
     uint32_t w[32];
-    quantize_p_units<8>(p, At, A, w, dump_codes, dump_step);
+    quantize_p_units<8>(p, At, A, w, dump_codes, dump_step, sum_out);
     const uint32_t row_base = p_sub_base + (row >> 3) * 1024 + (row & 7) * 128;
     const int sw = row & 7;
 #pragma unroll

@@ -23,6 +23,6 @@ cudaError_t launch_smooth_finalize(const float* kmax, const float* qmax, int S, 
 // Attention forward on the BF16 operand images; returns a hifa4_status.
 int launch_attention(const hifa4_shape& shape, const HeadMap& map, const hifa4_qkv& qkv,
                      const hifa4_attn_params& prm, void* out, const hifa4_debug* dbg,
-                     int* d_status, cudaStream_t st);
+                     const hifa4_mass_stats* stats, int* d_status, cudaStream_t st);
 
 }  // namespace hifa4

@@ -1,0 +1,122 @@
+"""GPU parity of the ablation modes of "P-Reordering": the mismatched normalizer (Theorem 1's
+O_mis: l accumulated from the unquantized FP16 P) and the histogram of the per-tile mass error
+eps = sum P-hat / sum P - 1, both against the CPU oracle through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_04302_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def hb():
+    from paper_2607_04302_b200 import binding
+    binding.lib()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def par():
+    from tests import parity
+    return parity
+
+
+CASES = {
+    "d128-bc64-causal-gqa": synth.config("C2", N=512, Hq=4, Hkv=2, cal_samples=4, cal_tokens=128),
+    "d128-bc128-ragged": synth.config("C2", N=320, Hq=2, Hkv=1, Bc=128, cal_samples=4, cal_tokens=128),
+    "d64-bc128-noncausal": synth.config("C3", N=256, Hq=2, Hkv=1, d=64, Bc=128, causal=False),
+    "d64-bc64-fp16": synth.config("C3", N=256, Hq=2, Hkv=1, d=64, Bc=64, dtype="fp16"),
+    "d256-bc64-mild": synth.config("C4", N=256, Hq=2, Hkv=1, Bc=64, cal_samples=3, cal_tokens=64),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_mismatched_normalizer_elementwise(hb, par, name):
+    cfg = CASES[name]
+    res = par.run_case(cfg, DEV, normalizer=1, check_quant=False)
+    print(par.assert_within_bars(res, name + " mismatched"))
+    assert res["rows"] == cfg.B * cfg.Hq * cfg.N
+
+
+def test_mismatched_differs_from_consistent_by_the_mass_error(hb, par):
+    """O_mis = O_con * (l_con / l_mis) row by row (same numerator, different denominators), and the
+    ratio is below 1 for nearly every row: HIF4 loses probability mass (Theorem 1, eps-bar < 0)."""
+    cfg = CASES["d128-bc64-causal-gqa"]
+    q, k, v = (t.to(DEV) for t in synth.make_qkv(cfg))
+    s, inv_s = par.calibrate(cfg, DEV)
+    qkv = hb.quantize_qkv(q, k, v, s, inv_s)
+    blocks = [(0, h, t) for h in range(cfg.Hq) for t in range(cfg.N // 128)]
+    o_con, d_con = hb.attention_fwd(qkv, True, Bc=64, debug_blocks=blocks)
+    o_mis, d_mis = hb.attention_fwd(qkv, True, Bc=64, debug_blocks=blocks, normalizer=1)
+    assert torch.equal(d_con["p_codes"], d_mis["p_codes"])
+    l_con = d_con["l"].reshape(cfg.Hq, cfg.N).half().float()
+    l_mis = d_mis["l"].reshape(cfg.Hq, cfg.N).half().float()
+    ratio = (l_con / l_mis)[None, :, :, None]
+    torch.testing.assert_close(o_mis, o_con * ratio, rtol=1e-5, atol=1e-6)
+    frac_loss = float((l_con < l_mis).float().mean())
+    assert frac_loss > 0.9, frac_loss
+
+
+def _oracle_eps(cfg, par, orc, q, k, v, s, inv_s, heads):
+    """eps per (row, key tile) from the oracle's P and P-hat dumps."""
+    dt = orc.F16 if cfg.dtype == "fp16" else orc.BF16
+    qn, kn, vn = par.np32(q), par.np32(k), par.np32(v)
+    s_np = None if s is None else par.np32(s)
+    is_np = None if inv_s is None else par.np32(inv_s)
+    eps = []
+    for b in range(cfg.B):
+        for h in heads:
+            g = h // (cfg.Hq // cfg.Hkv)
+            idx = np.arange(cfg.N, dtype=np.int32)
+            _, d = orc.attention_rows(qn[b, h], idx, kn[b, g], vn[b, g], None if s_np is None else s_np[g],
+                                      None if is_np is None else is_np[g], causal=cfg.causal, Bc=cfg.Bc,
+                                      in_dtype=dt, dumps=True)
+            nt = -(-cfg.N // cfg.Bc)
+            pad = nt * cfg.Bc - cfg.N
+            pr = np.pad(d["p_raw"], ((0, 0), (0, pad))).reshape(cfg.N, nt, cfg.Bc).sum(-1)
+            ph = np.pad(d["p_hat"], ((0, 0), (0, pad))).reshape(cfg.N, nt, cfg.Bc).sum(-1)
+            ok = pr > 0
+            eps.append(ph[ok] / pr[ok] - 1.0)
+    return np.concatenate(eps)
+
+
+@pytest.mark.parametrize("name", ["d128-bc64-causal-gqa", "d128-bc128-ragged", "d64-bc128-noncausal", "d256-bc64-mild"])
+def test_mass_error_histogram_matches_oracle(hb, par, name):
+    from oracle import hifa4_oracle as orc
+    cfg = CASES[name]
+    q, k, v = synth.make_qkv(cfg)
+    s, inv_s = par.calibrate(cfg, DEV)
+    qkv = hb.quantize_qkv(q.to(DEV), k.to(DEV), v.to(DEV), s, inv_s)
+    n_bins, lo, hi = 64, -0.16, 0.16
+    out, hist = hb.attention_fwd_stats(qkv, cfg.causal, n_bins, lo, hi, Bc=cfg.Bc)
+    torch.cuda.synchronize()
+    assert torch.equal(out, hb.attention_fwd(qkv, cfg.causal, Bc=cfg.Bc))      # statistics do not change the result
+    eps = _oracle_eps(cfg, par, orc, q, k, v, s, inv_s, range(cfg.Hq))
+    x = np.floor((eps - lo) * (n_bins / (hi - lo)))
+    ref = np.zeros(n_bins + 2, np.int64)
+    np.add.at(ref, np.where(x < 0, n_bins, np.where(x >= n_bins, n_bins + 1, x)).astype(np.int64), 1)
+    got = hist.cpu().numpy()
+    assert got.sum() == ref.sum() == eps.size                     # every (row, tile) pair with mass is counted once
+    # P differs from the oracle's only where ex2.approx and exp2 round to different FP16 values: a
+    # handful of pairs may sit in a neighbouring bin
+    assert np.abs(got - ref).sum() <= max(4, 2e-3 * eps.size), (got, ref)
+    centers = lo + (np.arange(n_bins) + 0.5) * (hi - lo) / n_bins
+    inside = got[:n_bins].sum()
+    assert inside > 0.95 * eps.size
+    mean_hist = float((got[:n_bins] * centers).sum() / inside)
+    assert mean_hist < 0 and abs(mean_hist - float(eps[(eps >= lo) & (eps < hi)].mean())) < 3e-3
+
+
+def test_stats_arguments_are_validated(hb, par):
+    cfg = synth.config("C3", N=64, Hq=1, Hkv=1)
+    q, k, v = (t.to(DEV) for t in synth.make_qkv(cfg))
+    qkv = hb.quantize_qkv(q, k, v)
+    with pytest.raises(hb.Hifa4Error):
+        hb.attention_fwd_stats(qkv, True, 0, -0.1, 0.1, Bc=64)
+    with pytest.raises(hb.Hifa4Error):
+        hb.attention_fwd_stats(qkv, True, 8, 0.1, -0.1, Bc=64)
+    with pytest.raises(hb.Hifa4Error):
+        hb.attention_fwd(qkv, True, Bc=64, normalizer=2)
