@@ -90,8 +90,8 @@ typedef struct {
 } hifa4_qkv;
 
 /* Calibration result summary (host memory).  rho_K and T_KQ are the gate
- * statistics of "Adaptive Applicability Gate"; they are NaN unless mode 3 is
- * built.  branch: 0 bypass, 1 strong, 2 mild, 4 caller's alpha. */
+ * statistics of "Adaptive Applicability Gate"; this struct reports them as NaN
+ * (hifa4_smooth_calibrate_auto computes them, into device memory).  branch: 0 bypass, 1 strong, 2 mild, 4 caller's alpha. */
 typedef struct { float rho_K, T_KQ; int branch; float alpha; } hifa4_calib_stats;
 
 /* Attention parameters.
@@ -161,7 +161,8 @@ void hifa4_get_counters(unsigned long long out[4]);
  *   combined by root-mean-square; s = Kagg^alpha / Qagg^(1-alpha), 1 where an
  *   aggregate is zero.  mode: 0 bypass (s = 1), 1 strong (alpha 0.5), 2 mild
  *   (alpha 0.25), 4 caller's alpha; 3 (gate decides) returns
- *   HIFA4_ERR_UNSUPPORTED.
+ *   HIFA4_ERR_UNSUPPORTED here: use hifa4_smooth_calibrate_auto, which takes
+ *   the extra scratch the gate statistics need.
  *   Outputs (device): s, inv_s [Hkv,d] floats, inv_s = fl32(1/s).
  *   absmax_ws: device scratch of 2*S*Hkv*d floats; the call clears it.
  *   host_stats: optional HOST struct, filled without synchronizing. */
@@ -169,6 +170,25 @@ int hifa4_smooth_calibrate(const void* q_cal, const void* k_cal, int S, int Hq, 
                            int Ncal, int d, const int* q_to_kv, int dt, int mode, float alpha,
                            float* s, float* inv_s, float* absmax_ws,
                            hifa4_calib_stats* host_stats, void* stream);
+
+/* Calibration with the applicability gate deciding the branch ("Adaptive Applicability
+ * Gate"), entirely on the device:
+ *   rho_K = max|K| / P99(|K|), the 99th percentile (nearest rank) over every element of
+ *   k_cal, read off an exact histogram of the 15-bit magnitude patterns;
+ *   T = max|K| / max|Q| over every element of k_cal and q_cal;
+ *   rho_K >= 6 and T >= 2 select Smooth-QK, with alpha = 0.5 (strong) if T > 3 and
+ *   alpha = 0.25 (mild) if 2 <= T <= 3; anything else bypasses (s = 1).
+ * Arguments as hifa4_smooth_calibrate, plus
+ *   gate_ws : device scratch of HIFA4_GATE_WS_BYTES bytes, 8-byte aligned;
+ *   d_stats : NULL, or DEVICE array of 4 floats that receives rho_K, T, the branch
+ *             (0 bypass, 1 strong, 2 mild) and alpha.  The call does not synchronize: copy
+ *             the four floats back after the stream has run if the host wants them.
+ * S*Hkv*Ncal*d must be below 2^32 (HIFA4_ERR_UNSUPPORTED otherwise). */
+#define HIFA4_GATE_WS_BYTES (32768u * 4u + 64u)
+int hifa4_smooth_calibrate_auto(const void* q_cal, const void* k_cal, int S, int Hq, int Hkv,
+                                int Ncal, int d, const int* q_to_kv, int dt, float* s,
+                                float* inv_s, float* absmax_ws, void* gate_ws, float* d_stats,
+                                void* stream);
 
 /* hifa4_smooth_calibrate for callers that cannot allocate device memory.
  * (The paper has no counterpart: this entry point exists for deployment only.)

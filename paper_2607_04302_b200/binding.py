@@ -89,6 +89,10 @@ def lib():
                                              C.c_int, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_float,
                                              C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(_CalibStats),
                                              C.c_void_p]
+        L.hifa4_smooth_calibrate_auto.restype = C.c_int
+        L.hifa4_smooth_calibrate_auto.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
+                                                  C.c_int, C.POINTER(C.c_int), C.c_int, C.c_void_p, C.c_void_p,
+                                                  C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.hifa4_smooth_calibrate_static.restype = C.c_int
         L.hifa4_smooth_calibrate_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int,
                                                     C.c_int, C.POINTER(C.c_int), C.c_int, C.c_int, C.c_float,
@@ -114,7 +118,7 @@ def lib():
 STATIC_CALIB_MAX_FLOATS = 1 << 20
 
 EXPORTS = ("hifa4_status_string", "hifa4_get_counters", "hifa4_smooth_calibrate",
-           "hifa4_smooth_calibrate_static", "hifa4_quant_bytes",
+           "hifa4_smooth_calibrate_static", "hifa4_smooth_calibrate_auto", "hifa4_quant_bytes",
            "hifa4_quantize_qkv", "hifa4_attention_workspace_bytes", "hifa4_attention_fwd",
            "hifa4_attention_fwd_stats", "hifa4_attention_raw_workspace_bytes", "hifa4_attention_fwd_raw")
 
@@ -232,6 +236,28 @@ def smooth_calibrate(q_cal, k_cal, mode, alpha=0.0, q_to_kv=None):
                                       C.byref(stats), _stream())
     _check(rc, "hifa4_smooth_calibrate")
     return s, inv_s
+
+
+GATE_WS_BYTES = 32768 * 4 + 64
+
+
+def smooth_calibrate_auto(q_cal, k_cal, q_to_kv=None):
+    """Calibration with the applicability gate deciding the branch on the device.
+    Returns (s, inv_s, stats) with stats a DEVICE float32 tensor [rho_K, T_K/Q, branch, alpha]."""
+    assert q_cal.is_cuda and k_cal.is_cuda and q_cal.is_contiguous() and k_cal.is_contiguous()
+    S, Hq, Ncal, d = q_cal.shape
+    Hkv = k_cal.shape[1]
+    dev = q_cal.device
+    s = torch.empty((Hkv, d), dtype=torch.float32, device=dev)
+    inv_s = torch.empty_like(s)
+    ws = torch.empty((2, S, Hkv, d), dtype=torch.float32, device=dev)
+    gate_ws = torch.empty(GATE_WS_BYTES // 8, dtype=torch.int64, device=dev)
+    stats = torch.zeros(4, dtype=torch.float32, device=dev)
+    keep, mp = _map_arr(q_to_kv)
+    rc = lib().hifa4_smooth_calibrate_auto(_ptr(q_cal), _ptr(k_cal), S, Hq, Hkv, Ncal, d, mp, _DT[q_cal.dtype],
+                                           _ptr(s), _ptr(inv_s), _ptr(ws), _ptr(gate_ws), _ptr(stats), _stream())
+    _check(rc, "hifa4_smooth_calibrate_auto")
+    return s, inv_s, stats
 
 
 def smooth_calibrate_static(q_cal, k_cal, mode, alpha=0.0, q_to_kv=None, s=None, inv_s=None):

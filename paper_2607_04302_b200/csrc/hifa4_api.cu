@@ -102,7 +102,7 @@ int hifa4_smooth_calibrate(const void* q_cal, const void* k_cal, int S, int Hq, 
         if (launch_absmax(dt, k_cal, kmap, S, Hkv, Hkv, Ncal, d, kmax, st) != cudaSuccess) return HIFA4_ERR_CUDA;
         if (launch_absmax(dt, q_cal, qmap, S, Hq, Hkv, Ncal, d, qmax, st) != cudaSuccess) return HIFA4_ERR_CUDA;
     }
-    if (launch_smooth_finalize(kmax, qmax, S, Hkv * d, a, mode == 0, s, inv_s, st) != cudaSuccess)
+    if (launch_smooth_finalize(kmax, qmax, S, Hkv * d, a, mode == 0, nullptr, s, inv_s, st) != cudaSuccess)
         return HIFA4_ERR_CUDA;
     if (host_stats) {
         host_stats->rho_K = NAN;
@@ -110,6 +110,35 @@ int hifa4_smooth_calibrate(const void* q_cal, const void* k_cal, int S, int Hq, 
         host_stats->branch = mode;
         host_stats->alpha = (float)a;
     }
+    return HIFA4_OK;
+}
+
+int hifa4_smooth_calibrate_auto(const void* q_cal, const void* k_cal, int S, int Hq, int Hkv, int Ncal,
+                                int d, const int* q_to_kv, int dt, float* s, float* inv_s, float* absmax_ws,
+                                void* gate_ws, float* d_stats, void* stream)
+{
+    g_calls[0].fetch_add(1, std::memory_order_relaxed);
+    if (!q_cal || !k_cal || !s || !inv_s || !absmax_ws || !gate_ws) return HIFA4_ERR_INVALID_ARG;
+    if (S <= 0 || Ncal <= 0) return HIFA4_ERR_INVALID_ARG;
+    if (dt != HIFA4_F16 && dt != HIFA4_BF16) return HIFA4_ERR_INVALID_ARG;
+    if (d != 64 && d != 128 && d != 256) return HIFA4_ERR_UNSUPPORTED;
+    if (((uintptr_t)gate_ws & 7u) != 0) return HIFA4_ERR_INVALID_ARG;
+    HeadMap qmap, kmap;
+    int rc = build_map(Hq, Hkv, q_to_kv, qmap, kmap);
+    if (rc) return rc;
+    const long long nk = (long long)S * Hkv * Ncal * d;
+    if (nk >= (1ll << 32)) return HIFA4_ERR_UNSUPPORTED;          // 32-bit histogram counters
+    if ((rc = check_arch())) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t n = (size_t)S * Hkv * d;
+    float* kmax = absmax_ws;
+    float* qmax = absmax_ws + n;
+    if (cudaMemsetAsync(absmax_ws, 0, 2 * n * sizeof(float), st) != cudaSuccess) return HIFA4_ERR_CUDA;
+    if (launch_absmax(dt, k_cal, kmap, S, Hkv, Hkv, Ncal, d, kmax, st) != cudaSuccess) return HIFA4_ERR_CUDA;
+    if (launch_absmax(dt, q_cal, qmap, S, Hq, Hkv, Ncal, d, qmax, st) != cudaSuccess) return HIFA4_ERR_CUDA;
+    if (launch_gate(dt, k_cal, nk, kmax, qmax, (int)n, gate_ws, d_stats, st) != cudaSuccess) return HIFA4_ERR_CUDA;
+    if (launch_smooth_finalize(kmax, qmax, S, Hkv * d, 0.0, 0, gate_result(gate_ws), s, inv_s, st) != cudaSuccess)
+        return HIFA4_ERR_CUDA;
     return HIFA4_OK;
 }
 

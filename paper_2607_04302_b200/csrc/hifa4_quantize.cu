@@ -283,12 +283,14 @@ absmax_kernel(const uint16_t* __restrict__ x, HeadMap map, int H, int Hkv, int N
 }
 
 // s = Kagg^alpha / Qagg^(1-alpha) with RMS aggregation over samples; 1 where degenerate.
+// gate (optional, device): {alpha, bypass flag} chosen by the applicability gate; overrides the arguments.
 __global__ void smooth_finalize_kernel(const float* __restrict__ kmax, const float* __restrict__ qmax,
-                                       int S, int n, double alpha, int bypass, float* __restrict__ s,
-                                       float* __restrict__ inv_s)
+                                       int S, int n, double alpha, int bypass, const double* __restrict__ gate,
+                                       float* __restrict__ s, float* __restrict__ inv_s)
 {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
+    if (gate) { alpha = gate[0]; bypass = gate[1] != 0.0; }
     double ks = 0, qs = 0;
     for (int m = 0; m < S; ++m) {
         double a = kmax[(long long)m * n + i], b = qmax[(long long)m * n + i];
@@ -346,9 +348,9 @@ cudaError_t launch_absmax(int dtype, const void* x, const HeadMap& map, int S, i
 }
 
 cudaError_t launch_smooth_finalize(const float* kmax, const float* qmax, int S, int n, double alpha,
-                                   int bypass, float* s, float* inv_s, cudaStream_t st)
+                                   int bypass, const double* gate, float* s, float* inv_s, cudaStream_t st)
 {
-    smooth_finalize_kernel<<<(n + 127) / 128, 128, 0, st>>>(kmax, qmax, S, n, alpha, bypass, s, inv_s);
+    smooth_finalize_kernel<<<(n + 127) / 128, 128, 0, st>>>(kmax, qmax, S, n, alpha, bypass, gate, s, inv_s);
     count_launch();
     return cudaGetLastError();
 }
