@@ -201,6 +201,8 @@ def main():
     ap.add_argument("--workload", default="C2", help="C2 (headline), C3, C4, C5 or C5@<N>")
     ap.add_argument("--noncausal", action="store_true")
     ap.add_argument("--Bc", type=int, default=0, help="key-tile width (default: the configuration's, 64)")
+    ap.add_argument("--p-f32", action="store_true",
+                    help="variant: quantize the FP32 exponential (not the method's FP16 P; for comparison only)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -257,7 +259,8 @@ def main():
         hb.quantize_qkv(q, k, v, s, inv_s, out=qkv, d_status=status)
         mid = torch.cuda.Event(enable_timing=True)
         mid.record()
-        hb.attention_fwd(qkv, cfg.causal, Bc=cfg.Bc, out_dtype=hb.F32, out=out, d_status=status)
+        hb.attention_fwd(qkv, cfg.causal, Bc=cfg.Bc, out_dtype=hb.F32, out=out, d_status=status,
+                         p_dtype=hb.F32 if args.p_f32 else hb.F16)
         return mid
 
     def barrier():
@@ -373,6 +376,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "N": cfg.N, "d": cfg.d,
                        "causal": cfg.causal, "Br": 128, "Bc": cfg.Bc, "in_dtype": cfg.dtype, "out_dtype": "f32",
+                       "p_dtype": "f32 (variant)" if args.p_f32 else "f16",
                        "smooth_mode": cfg.smooth_mode, "step": "hifa4_quantize_qkv + hifa4_attention_fwd",
                        "l2": "flushed between steps (256 MiB write), outside the per-step events",
                        "parallelism": f"replicated batches x{world}"},

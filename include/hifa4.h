@@ -111,6 +111,10 @@ typedef struct { float rho_K, T_KQ; int branch; float alpha; } hifa4_calib_stats
  *               hifa4_quantize_qkv.  0: no correction (the Q buffers must then hold un-centred Q).
  *   p_dtype     HIFA4_F16: exp(S-m) is rounded to FP16 before quantization
  *               ("FP16 operations", Appendix "Implementation Details").
+ *               HIFA4_F32: variant that quantizes the FP32 exponential directly (a
+ *               different function: it changes a few 1e-4 of the P-hat codes); built
+ *               for Bc = 64 with d = 128 or 256 and the consistent normalizer,
+ *               HIFA4_ERR_UNSUPPORTED elsewhere.
  *   out_dtype   HIFA4_F16 / HIFA4_BF16 / HIFA4_F32 element type of `out`.
  *   softmax_scale  0 selects 1/sqrt(d). */
 typedef struct {

@@ -300,13 +300,14 @@ def quantize_qkv(q, k, v, s=None, inv_s=None, q_to_kv=None, out: QuantizedQKV | 
 
 
 def attention_fwd(qkv: QuantizedQKV, causal: bool, Bc: int = 128, out_dtype=F32, out=None,
-                  debug_blocks=None, d_status=None, softmax_scale=0.0, Br=128, qmean=False, normalizer=0):
+                  debug_blocks=None, d_status=None, softmax_scale=0.0, Br=128, qmean=False, normalizer=0,
+                  p_dtype=F16):
     """Fused attention forward on quantized operands.  Returns out [B,Hq,N,d], or
     (out, dict(p_codes, p_step, l, m)) when debug_blocks (a list of (b, h, query block)) is given."""
     dev = qkv.q_mma.device
     sh = _shape(qkv.B, qkv.Hq, qkv.Hkv, qkv.N, qkv.d, qkv.in_dtype, qkv.q_to_kv)
     prm = _params(causal, Bc, out_dtype, Br=Br, softmax_scale=softmax_scale, qmean=int(qmean),
-                  normalizer=int(normalizer))
+                  normalizer=int(normalizer), p_dtype=p_dtype)
     if out is None:
         out = torch.empty((qkv.B, qkv.Hq, qkv.N, qkv.d), dtype=_TORCH_DT[out_dtype], device=dev)
     st = qkv.struct()

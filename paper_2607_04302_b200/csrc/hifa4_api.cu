@@ -190,7 +190,8 @@ static int check_attn(const hifa4_shape* shape, const hifa4_attn_params* prm)
     if (shape->d == 256 && prm->Bc != 64) return HIFA4_ERR_UNSUPPORTED;
     if (prm->qmean != 0 && prm->qmean != 1) return HIFA4_ERR_INVALID_ARG;
     if (prm->normalizer != 0 && prm->normalizer != 1) return HIFA4_ERR_INVALID_ARG;
-    if (prm->p_dtype != HIFA4_F16) return HIFA4_ERR_UNSUPPORTED;
+    if (prm->p_dtype != HIFA4_F16 && prm->p_dtype != HIFA4_F32) return HIFA4_ERR_INVALID_ARG;
+    if (prm->p_dtype == HIFA4_F32 && (prm->Bc != 64 || shape->d == 64 || prm->normalizer)) return HIFA4_ERR_UNSUPPORTED;
     return HIFA4_OK;
 }
 

@@ -367,6 +367,11 @@ int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv&
         a.dbg.l_out = dbg->l_out; a.dbg.m_out = dbg->m_out;
     }
     a.normalizer = prm.normalizer ? 1 : 0;
+    a.p_f32 = prm.p_dtype == HIFA4_F32 ? 1 : 0;
+    if (a.p_f32) {                                // variant built for the 64-key warp-specialised kernels only
+        if (a.normalizer || stats || prm.Bc != 64 || (sh.d != 128 && sh.d != 256)) return HIFA4_ERR_UNSUPPORTED;
+        return launch_attention_ws64(sh, qkv, a, st);
+    }
     if (stats) {
         a.hist = stats->hist;
         a.n_bins = stats->n_bins;

@@ -28,6 +28,7 @@ struct AttnArgs {
     unsigned long long* hist;     // mass-error histogram [n_bins + 2] or null
     int n_bins;
     double hist_lo, hist_inv_w;   // bin = floor((eps - lo) * inv_w)
+    int p_f32;                    // keep P in FP32 before quantization (variant; default FP16)
     int qmean;                    // add mu_i * k_sum_j to the raw scores (Algorithm 1 line 6)
     const float* q_mu;            // [B,Hq,N]
     const float* k_sum;           // [B,Hkv,N]
@@ -145,9 +146,11 @@ __device__ __forceinline__ void quantize_p_units(const float (&p)[NU * 8], const
 // the group maximum of the accumulators through the same instruction sequence
 // (p_of_score): that is exact because fma, ex2.approx (checked exhaustively over [-40, 0]) and
 // the FP16 rounding are all monotone non-decreasing.
+template <bool PF32 = false>
 __device__ __forceinline__ float p_of_score(float acc, float c1, float mL)
 {
-    return f16_round(ex2_approx(fmaf(acc, c1, -mL)));
+    const float e = ex2_approx(fmaf(acc, c1, -mL));
+    return PF32 ? e : f16_round(e);                    // PF32: the variant that keeps P in FP32
 }
 
 // Arithmetic of the fused form (all exact except the exponential itself):
@@ -185,34 +188,35 @@ __device__ __forceinline__ PQuantConst p_quant_const(float c1, float mL, float A
     return k;
 }
 
-// P = exp2(acc * c1 - mL) rounded to FP16 for the 8 keys of unit u.
-template <int NU>
+// P = exp2(acc * c1 - mL) rounded to FP16 (PF32: left in FP32) for the 8 keys of unit u.
+template <int NU, bool PF32 = false>
 __device__ __forceinline__ void exp_unit(const float (&acc)[NU * 8], int u, const PQuantConst& k, float (&p)[8])
 {
 #pragma unroll
     for (int i = 0; i < 8; i += 2) {
         float t0, t1;
         unpack2(fma2(pack2(acc[8 * u + i], acc[8 * u + i + 1]), k.c1c1, k.nml), t0, t1);
-        exp2_f16_pair(t0, t1, p[i], p[i + 1]);
+        if (PF32) { p[i] = ex2_approx(t0); p[i + 1] = ex2_approx(t1); }
+        else exp2_f16_pair(t0, t1, p[i], p[i + 1]);
     }
 }
 
 // Units U0..U1-1 of a thread's NU units: acc -> P (FP16) -> P-hat image words w[4u..4u+3].
 // The exponentials of unit u+1 are issued before unit u is quantized, so that the MUFU latency of
 // one unit hides behind the ALU/FMA work of the previous one.
-template <int NU, int U0, int U1, bool DBG>
+template <int NU, int U0, int U1, bool DBG, bool PF32 = false>
 __device__ __forceinline__ void exp_quantize_units(const float (&acc)[NU * 8], const PQuantConst& k, bool zero_group,
                                                    uint32_t (&w)[NU * 4], uint8_t* dump_codes, float* dump_step)
 {
     const uint32_t MAGIC_BITS = 0x4B400000u;                               // 1.5 * 2^23
     float pn[8];
-    exp_unit<NU>(acc, U0, k, pn);
+    exp_unit<NU, PF32>(acc, U0, k, pn);
 #pragma unroll
     for (int u = U0; u < U1; ++u) {
         float p[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) p[i] = pn[i];
-        if (u + 1 < U1) exp_unit<NU>(acc, u + 1, k, pn);
+        if (u + 1 < U1) exp_unit<NU, PF32>(acc, u + 1, k, pn);
         const float At0 = fmaxf(max3(p[0], p[1], p[2]), p[3]);
         const float At1 = fmaxf(max3(p[4], p[5], p[6]), p[7]);
         const int n0 = max((int)__float_as_uint(At0) + k.tadd, 0) >> 23;

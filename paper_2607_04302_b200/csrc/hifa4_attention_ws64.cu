@@ -64,7 +64,7 @@ static __device__ __forceinline__ bool wait64(uint32_t bar, uint32_t parity, vol
     return false;
 }
 
-template <int DH, bool DBG>
+template <int DH, bool DBG, bool PF32>
 __global__ void __launch_bounds__(WS64<DH>::THREADS, WS64<DH>::CTAS_PER_SM)
 attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                            const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnArgs args)
@@ -306,7 +306,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             if (jt > 0 && m_new != m_run) rsc = f16_round(ex2_approx((m_run - m_new) * LOG2E));
             m_run = m_new;
             const float mL = m_run * LOG2E;
-            const float A = p_of_score(mx, args.c1, mL);       // = max of P over the group (monotone map)
+            const float A = p_of_score<PF32>(mx, args.c1, mL); // = max of P over the group (monotone map)
 
             // P = exp(S - m) in FP16 (line 9), P-hat = HIF4(P) (line 10)
             uint8_t* dc = nullptr;
@@ -318,7 +318,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             }
             uint32_t w[NU * 4];
             const PQuantConst qc = p_quant_const(args.c1, mL, A);
-            exp_quantize_units<NU, 0, NU, DBG>(p, qc, A == 0.f, w, dc, ds);
+            exp_quantize_units<NU, 0, NU, DBG, PF32>(p, qc, A == 0.f, w, dc, ds);
             // the P-hat columns and [O | l] are free once PV(jt-1) has completed (every warp observes
             // every phase of that barrier, in order)
             if (jt > 0) {
@@ -451,7 +451,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     if (warp == W_MMA) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
 }
 
-template <int DH, bool DBG>
+template <int DH, bool DBG, bool PF32>
 static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
     using C = WS64<DH>;
@@ -459,7 +459,7 @@ static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnAr
     if (!make_bf16_map(&mq, qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, DH, 128)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, DH, C::BC)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, DH, sh.N, DH)) return HIFA4_ERR_CUDA;
-    auto kern = attention_fwd_ws64_kernel<DH, DBG>;
+    auto kern = attention_fwd_ws64_kernel<DH, DBG, PF32>;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
@@ -475,8 +475,13 @@ static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnAr
 int launch_attention_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
     const bool dbg = args.dbg.n_blocks > 0;
-    if (sh.d == 256) return dbg ? launch_ws64<256, true>(sh, qkv, args, st) : launch_ws64<256, false>(sh, qkv, args, st);
-    if (sh.d == 128) return dbg ? launch_ws64<128, true>(sh, qkv, args, st) : launch_ws64<128, false>(sh, qkv, args, st);
+    if (args.p_f32) {
+        if (sh.d == 256) return dbg ? launch_ws64<256, true, true>(sh, qkv, args, st) : launch_ws64<256, false, true>(sh, qkv, args, st);
+        if (sh.d == 128) return dbg ? launch_ws64<128, true, true>(sh, qkv, args, st) : launch_ws64<128, false, true>(sh, qkv, args, st);
+        return HIFA4_ERR_UNSUPPORTED;
+    }
+    if (sh.d == 256) return dbg ? launch_ws64<256, true, false>(sh, qkv, args, st) : launch_ws64<256, false, false>(sh, qkv, args, st);
+    if (sh.d == 128) return dbg ? launch_ws64<128, true, false>(sh, qkv, args, st) : launch_ws64<128, false, false>(sh, qkv, args, st);
     return HIFA4_ERR_UNSUPPORTED;
 }
 

@@ -69,7 +69,7 @@ def check_quantized(cfg, q, k, v, s, inv_s, qkv, qmean=False):
 
 
 def run_case(cfg, device="cuda:0", blocks=None, out_dtype=hb.F32, check_quant=True, rows_per_block=None,
-             qkv_host=None, qmean=False, normalizer=0):
+             qkv_host=None, qmean=False, normalizer=0, p_dtype=hb.F16):
     """Full path on the GPU + oracle on the requested 128-row query blocks.
 
     blocks: list of (b, h, query_block); default: every block (small cases only).
@@ -90,7 +90,7 @@ def run_case(cfg, device="cuda:0", blocks=None, out_dtype=hb.F32, check_quant=Tr
     for i0 in range(0, len(blocks), hb.MAX_DEBUG_BLOCKS):
         chunk = blocks[i0:i0 + hb.MAX_DEBUG_BLOCKS]
         out, dump = hb.attention_fwd(qkv, cfg.causal, Bc=cfg.Bc, out_dtype=out_dtype, debug_blocks=chunk,
-                                     d_status=status, qmean=qmean, normalizer=normalizer)
+                                     d_status=status, qmean=qmean, normalizer=normalizer, p_dtype=p_dtype)
         torch.cuda.synchronize()
         assert int(status.item()) == 0, f"device status {int(status.item())}"
         out_full = out
@@ -109,7 +109,7 @@ def run_case(cfg, device="cuda:0", blocks=None, out_dtype=hb.F32, check_quant=Tr
             o_ref, d = orc.attention_rows(qn[b, h, idx], idx, kn[b, g], vn[b, g],
                                           None if s_np is None else s_np[g], None if is_np is None else is_np[g],
                                           causal=cfg.causal, Bc=cfg.Bc, in_dtype=dt, out_dtype=out_dtype,
-                                          qmean=int(qmean), normalizer=normalizer, dumps=True)
+                                          qmean=int(qmean), normalizer=normalizer, p_dtype=p_dtype, dumps=True)
             loc = idx - r0
             code_ne = pc[bi, loc] != d["p_codes"]
             step_ne = np.repeat(ps[bi, loc] != d["p_step"], 4, axis=1)

@@ -53,7 +53,7 @@ def test_size_queries_and_validation_without_gpu(lib):
     assert lib.hifa4_attention_fwd(C.byref(sh), C.byref(st), C.byref(prm), one, None, None, None, None) == 1
     prm = hb._params(True, 128, hb.F32, normalizer=2)                               # no such normaliser mode
     assert lib.hifa4_attention_fwd(C.byref(sh), C.byref(st), C.byref(prm), one, None, None, None, None) == 1
-    prm = hb._params(True, 128, hb.F32, p_dtype=hb.F32)                             # FP32 P: not built
+    prm = hb._params(True, 128, hb.F32, p_dtype=hb.F32)                             # FP32 P: built for 64-key tiles only
     assert lib.hifa4_attention_fwd(C.byref(sh), C.byref(st), C.byref(prm), one, None, None, None, None) == 2
     prm = hb._params(True, 128, hb.F32)                                             # histogram request without bins
     assert lib.hifa4_attention_fwd_stats(C.byref(sh), C.byref(st), C.byref(prm), one, None, None, None, None) == 1

@@ -120,3 +120,28 @@ def test_stats_arguments_are_validated(hb, par):
         hb.attention_fwd_stats(qkv, True, 8, 0.1, -0.1, Bc=64)
     with pytest.raises(hb.Hifa4Error):
         hb.attention_fwd(qkv, True, Bc=64, normalizer=2)
+
+
+PF32 = {
+    "d128-bc64-causal-gqa": CASES["d128-bc64-causal-gqa"],
+    "d128-bc64-ragged-noncausal": synth.config("C2", N=320, Hq=2, Hkv=1, causal=False, cal_samples=4, cal_tokens=128),
+    "d256-bc64-mild": CASES["d256-bc64-mild"],
+}
+
+
+@pytest.mark.parametrize("name", list(PF32))
+def test_fp32_p_variant_elementwise(hb, par, name):
+    """The variant that quantizes the FP32 exponential without the FP16 rounding of P, against the
+    oracle run with the same flag; it is a different function from the default."""
+    cfg = PF32[name]
+    res = par.run_case(cfg, DEV, p_dtype=hb.F32, check_quant=False)
+    print(par.assert_within_bars(res, name + " p=f32"))
+    ref = par.run_case(cfg, DEV, check_quant=False)
+    assert not torch.equal(res["out"], ref["out"])
+
+
+def test_fp32_p_variant_full_size_sampled(hb, par):
+    cfg = synth.config("C2")
+    blocks = [(0, h, t) for h in (0, 31) for t in (0, 15, 31)]
+    res = par.run_case(cfg, DEV, blocks=blocks, rows_per_block=16, check_quant=False, p_dtype=hb.F32)
+    print(par.assert_within_bars(res, "C2 p=f32"))
