@@ -528,35 +528,53 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 if (args.dbg.m_out) args.dbg.m_out[dbg_slot * 128 + r_loc] = m_run;
             }
             const size_t orow = ((size_t)bh_q * N + row) * D + kq * (D / KS);
+            // FP32 output goes through a 32 x 32 transpose in shared memory (the K stages are idle by now:
+            // every load has landed and every MMA has completed), so that a warp stores four whole
+            // 128-byte lines per instruction instead of 32 pieces of 16 bytes.
+            const uint32_t stage = k_s + (uint32_t)warp * 4096u;
 #pragma unroll
             for (int cc = 0; cc < D / KS / 32; ++cc) {
                 uint32_t r[32];
                 tmem_ld32(t_lane + kq * (D / KS) + cc * 32, r);
                 tmem_wait_ld();
-                if (row < N) {
-                    float o[32];
+                float o[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) o[i] = __fdiv_rn(__uint_as_float(r[i]), l16);
-                    if (args.out_dtype == HIFA4_F32) {
-                        float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.out) + orow + cc * 32);
+                for (int i = 0; i < 32; ++i) o[i] = __fdiv_rn(__uint_as_float(r[i]), l16);
+                if (args.out_dtype == HIFA4_F32) {
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
-                    } else {
-                        uint32_t w[16];
+                    for (int c4 = 0; c4 < 8; ++c4)
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};"
+                                     ::"r"(stage + lane * 128 + ((c4 ^ (lane & 7)) << 4)), "f"(o[4 * c4]), "f"(o[4 * c4 + 1]),
+                                       "f"(o[4 * c4 + 2]), "f"(o[4 * c4 + 3]) : "memory");
+                    __syncwarp();
+                    const int c4 = lane & 7;
+                    float* obase = reinterpret_cast<float*>(args.out) + ((size_t)bh_q * N + q0 + quarter * 32) * D +
+                                   kq * (D / KS) + cc * 32 + c4 * 4;
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            if (args.out_dtype == HIFA4_F16) {
-                                __half2 t = __floats2half2_rn(o[2 * i], o[2 * i + 1]);
-                                w[i] = *reinterpret_cast<uint32_t*>(&t);
-                            } else {
-                                __nv_bfloat162 t = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
-                                w[i] = *reinterpret_cast<uint32_t*>(&t);
-                            }
-                        }
-                        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(args.out) + orow + cc * 32);
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+                    for (int it = 0; it < 8; ++it) {
+                        const int rr = it * 4 + (lane >> 3);
+                        float4 v;
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                     : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                                     : "r"(stage + rr * 128 + ((c4 ^ (rr & 7)) << 4)));
+                        if (q0 + quarter * 32 + rr < N) *reinterpret_cast<float4*>(obase + (size_t)rr * D) = v;
                     }
+                    __syncwarp();
+                } else if (row < N) {
+                    uint32_t w[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        if (args.out_dtype == HIFA4_F16) {
+                            __half2 t = __floats2half2_rn(o[2 * i], o[2 * i + 1]);
+                            w[i] = *reinterpret_cast<uint32_t*>(&t);
+                        } else {
+                            __nv_bfloat162 t = __floats2bfloat162_rn(o[2 * i], o[2 * i + 1]);
+                            w[i] = *reinterpret_cast<uint32_t*>(&t);
+                        }
+                    }
+                    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(args.out) + orow + cc * 32);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
                 }
             }
         } else if (ok) {
