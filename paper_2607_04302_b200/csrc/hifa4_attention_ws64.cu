@@ -76,11 +76,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     constexpr int Q_BYTES = C::Q_BYTES, K_SUB = C::K_SUB, K_STAGE = C::K_STAGE, V_STAGE = C::V_STAGE;
     constexpr int O_COLS = C::O_COLS, QT_COL = C::QT_COL, S_COL = C::S_COL, P_COL = C::P_COL, TMEM_COLS = C::TMEM_COLS;
     if (args.d_status && *reinterpret_cast<volatile int*>(args.d_status) != 0) return;
-#ifdef HIFA4_PHASE_TIMING
-    const unsigned t_kernel_start = (unsigned)clock();
-    unsigned long long gt_start;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt_start));
-#endif
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -147,25 +142,13 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
                 const int j0 = jt * BC;
                 if (!wait64(bar(BAR_KE + st), ph ^ 1u, abort_flag)) { fail(1); break; }
-#ifdef HIFA4_PROBE_SKIP_K
-                if (jt >= 2) mbar_arrive(bar(BAR_KF + st)); else {
-#endif
                 mbar_expect_tx(bar(BAR_KF + st), K_STAGE);
 #pragma unroll
                 for (int s = 0; s < QSUB; ++s)
                     tma_load_3d(k_s + st * K_STAGE + s * K_SUB, &tmap_k, bar(BAR_KF + st), 64 * s, j0, bh_kv);
-#ifdef HIFA4_PROBE_SKIP_K
-                }
-#endif
                 if (!wait64(bar(BAR_VE + st), ph ^ 1u, abort_flag)) { fail(2); break; }
-#ifdef HIFA4_PROBE_SKIP_V
-                if (jt >= 2) mbar_arrive(bar(BAR_VF + st)); else {
-#endif
                 mbar_expect_tx(bar(BAR_VF + st), D * 128);
                 tma_load_3d(v_s + st * V_STAGE, &tmap_v, bar(BAR_VF + st), j0, 0, bh_kv);
-#ifdef HIFA4_PROBE_SKIP_V
-                }
-#endif
             }
         }
     } else if (warp == W_MMA) {
@@ -193,29 +176,17 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         };
         ok = wait64(bar(C::Q_IN_TMEM ? BAR_QT : BAR_Q), 0, abort_flag) && wait64(bar(BAR_KF), 0, abort_flag);
         if (ok) { tc_fence_after(); issue_qk(0); } else if (leader) fail(3);
-#ifdef HIFA4_PHASE_TIMING
-        unsigned mph[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        unsigned mprev = (unsigned)clock();
-#define MPHASE(i) { const unsigned tnow = (unsigned)clock(); mph[i] += tnow - mprev; mprev = tnow; }
-#else
-#define MPHASE(i)
-#endif
         for (int jt = 0; ok && jt < n_tiles; ++jt) {
             const int st = jt & 1;
             const uint32_t ph = (uint32_t)(jt >> 1) & 1u, par = (uint32_t)jt & 1u;
             if (jt + 1 < n_tiles) {                       // S(jt+1) as soon as S(jt) sits in registers
                 if (!wait64(bar(BAR_KF + (st ^ 1)), (uint32_t)((jt + 1) >> 1) & 1u, abort_flag)) { if (leader) fail(4); break; }
-                MPHASE(0)
                 if (!wait64(bar(BAR_SFREE), par, abort_flag)) { if (leader) fail(5); break; }
-                MPHASE(1)
                 tc_fence_after();
                 issue_qk(jt + 1);
-                MPHASE(2)
             }
             if (!wait64(bar(BAR_VF + st), ph, abort_flag)) { if (leader) fail(6); break; }
-            MPHASE(3)
             if (!wait64(bar(BAR_PF), par, abort_flag)) { if (leader) fail(7); break; }
-            MPHASE(4)
             tc_fence_after();
             const uint32_t b0 = v_lo + st * (V_STAGE >> 4);
             const uint32_t acc0 = jt > 0 ? 1u : 0u;
@@ -230,15 +201,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 umma_commit(bar(BAR_VE + st));
             }
             __syncwarp();
-            MPHASE(5)
         }
-#ifdef HIFA4_PHASE_TIMING
-        if (lane == 0 && args.q_mu && !args.qmean) {
-            float* tb = const_cast<float*>(args.q_mu) + (size_t)gridDim.x * 64 + (size_t)blockIdx.x * 8;
-            for (int i = 0; i < 6; ++i) tb[i] = (float)mph[i];
-            tb[7] = (float)n_tiles;
-        }
-#endif
     } else {
         // ------------------------------------------------------------------ softmax / quantize
         const int kq = warp >> 2, quarter = warp & 3;             // key half, row quarter
@@ -283,31 +246,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             } else { fail(13); ok = false; }
         }
 
-#ifdef HIFA4_PROBE_WAITLAT
-        if (args.q_mu && !args.qmean) {                  // latency of polls on a barrier whose phase is complete
-            wait64(bar(BAR_Q), 0, abort_flag);
-            const unsigned c0 = (unsigned)clock();
-            bool all = true;
-#pragma unroll 1
-            for (int i = 0; i < 16; ++i) all &= mbar_try_wait(bar(BAR_Q), 0);
-            const unsigned c1 = (unsigned)clock();
-            float acc = 0.f;
-#pragma unroll 1
-            for (int i = 0; i < 16; ++i) { xmax[(warp * 32 + lane) & 511] = acc; acc += xmax[(warp * 32 + lane + 1) & 511]; }
-            const unsigned c2 = (unsigned)clock();
-            if (lane == 0) {
-                float* tb = const_cast<float*>(args.q_mu) + ((size_t)blockIdx.x * 8 + warp) * 4;
-                tb[0] = (float)(c1 - c0) / 16.f; tb[1] = (float)(c2 - c1) / 16.f; tb[2] = all ? 1.f : 0.f; tb[3] = acc;
-            }
-        }
-#endif
-#ifdef HIFA4_PHASE_TIMING
-        unsigned tph[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        unsigned tprev = (unsigned)clock();
-#define PHASE(i) { const unsigned tnow = (unsigned)clock(); tph[i] += tnow - tprev; tprev = tnow; }
-#else
-#define PHASE(i)
-#endif
         bool sf_ready = false;
         for (int jt = 0; ok && jt < n_tiles; ++jt) {
             const int j0 = jt * BC;
@@ -315,7 +253,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             const int kbase = j0 + kq * KPT;
             // the poll for S(jt) was issued before the tail of the previous tile (a poll takes > 100 clk)
             if (!sf_ready && !wait64(bar(BAR_SF), par, abort_flag)) { fail(8); ok = false; break; }
-            PHASE(0)
             tc_fence_after();
             // The thread pulls its own KPT scores and, for the row maximum (line 7), the rest of the row
             // as well: the tile is one 64-key group, so row maximum = group maximum, and reading the other
@@ -393,7 +330,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                     for (int i = 0; i < w; ++i) t4[i] = fmaxf(t4[i], t4[i + w]);
                 mx = t4[0];
             }
-            PHASE(1)
 
             const float m_new = fmaxf(m_run, f16_round(mx * args.c0));
             float rsc = 1.f;
@@ -414,9 +350,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             const bool pv_ready = jt > 0 ? mbar_test_wait(bar(BAR_PV), par ^ 1u) : true;
             uint32_t w[NU * 4];
             const PQuantConst qc = p_quant_const(args.c1, mL, A);
-            PHASE(3)
             exp_quantize_units<NU, 0, NU, DBG, PF32>(p, qc, A == 0.f, w, dc, ds);
-            PHASE(4)
             // the P-hat columns and [O | l] are free once PV(jt-1) has completed (every warp observes
             // every phase of that barrier, in order)
             if (jt > 0) {
@@ -424,7 +358,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 tc_fence_after();
             }
             sf_ready = mbar_test_wait(bar(BAR_SF), par ^ 1u);   // S(jt+1): answer used at the top of the next tile
-            PHASE(5)
             if constexpr (NU == 8) tmem_st32(t_lane + P_COL, w);
             else if constexpr (NU == 4) tmem_st16(t_lane + P_COL + kq * (KPT / 2), w);
             else tmem_st8(t_lane + P_COL + kq * (KPT / 2), w);
@@ -505,15 +438,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_PF));
-            PHASE(6)
         }
-#ifdef HIFA4_PHASE_TIMING
-        if (lane == 0 && args.q_mu && !args.qmean) {
-            float* tb = const_cast<float*>(args.q_mu) + ((size_t)blockIdx.x * 8 + warp) * 8;
-            for (int i = 0; i < 7; ++i) tb[i] = (float)tph[i];
-            tb[7] = (float)n_tiles + 1e-4f * (float)tph[7];
-        }
-#endif
 
         // finalize: out = O / l with l rounded to FP16 (line 13); half kq writes channels (d/2)*kq..
         if (ok && wait64(bar(BAR_PV), (uint32_t)(n_tiles - 1) & 1u, abort_flag)) {
@@ -523,6 +448,10 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             tmem_wait_ld();
             const float ell = __uint_as_float(lr[0]);
             const float l16 = f16_round(ell);
+            // O / l as the correctly rounded quotient from the correctly rounded reciprocal: q0 = O * y,
+            // q = fma(fma(-q0, l, O), y, q0) (Markstein's correction step; no value here is near the ends of
+            // the FP32 range: l >= 2^-24 is an FP16 value and |O| <= l * max|V|)
+            const float rl = __frcp_rn(l16);
             if (DBG && dbg_slot >= 0 && row < N && kq == 0) {
                 if (args.dbg.l_out) args.dbg.l_out[dbg_slot * 128 + r_loc] = ell;
                 if (args.dbg.m_out) args.dbg.m_out[dbg_slot * 128 + r_loc] = m_run;
@@ -539,7 +468,11 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 tmem_wait_ld();
                 float o[32];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) o[i] = __fdiv_rn(__uint_as_float(r[i]), l16);
+                for (int i = 0; i < 32; ++i) {
+                    const float a = __uint_as_float(r[i]);
+                    const float q0 = a * rl;
+                    o[i] = fmaf(fmaf(-q0, l16, a), rl, q0);
+                }
                 if (args.out_dtype == HIFA4_F32) {
 #pragma unroll
                     for (int c4 = 0; c4 < 8; ++c4)
@@ -584,17 +517,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
 
     tc_fence_before();
     __syncthreads();
-#ifdef HIFA4_PHASE_TIMING
-    if (tid == 0 && args.q_mu && !args.qmean) {
-        const_cast<float*>(args.q_mu)[(size_t)gridDim.x * 64 + (size_t)blockIdx.x * 8 + 6] = (float)((unsigned)clock() - t_kernel_start);
-        unsigned long long gt_end;
-        unsigned smid;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt_end));
-        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-        unsigned long long* g = reinterpret_cast<unsigned long long*>(const_cast<float*>(args.q_mu) + (size_t)gridDim.x * 72) + (size_t)blockIdx.x * 3;
-        g[0] = gt_start; g[1] = gt_end; g[2] = smid;
-    }
-#endif
     if (warp == W_MMA) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
 }
 
