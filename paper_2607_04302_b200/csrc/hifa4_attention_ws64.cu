@@ -2,8 +2,9 @@
 //
 // One CTA = 128 query rows of one (batch, query head), 10 warps:
 //   warps 0-7  softmax / quantize: warp w owns rows 32*(w%4).. of the tile and keys 32*(w/4).. of
-//              every 64-key tile, i.e. half of the tile's single HIF4 group per thread; the two
-//              threads of a row exchange their partial score maxima through shared memory
+//              every 64-key tile, i.e. half of the tile's single HIF4 group per thread; for the row
+//              maximum each thread also reads the other half of its row from tensor memory (cheaper
+//              than an exchange between the two threads: a poll of an mbarrier costs > 100 clk)
 //   warp 8     TMA producer: Q once, then K and V^T tiles through two-stage rings
 //   warp 9     tcgen05 issuer
 // S has a single buffer that is released early: the softmax warps pull S(j) into registers and
@@ -37,8 +38,7 @@ struct WS64 {
     static constexpr int K_OFF = Q_OFF + Q_BYTES;
     static constexpr int V_OFF = K_OFF + STAGES * K_STAGE;
     static constexpr int MISC_OFF = V_OFF + STAGES * V_STAGE;
-    static constexpr int XCHG_OFF = MISC_OFF + 256;         // partial row maxima [2 parities][2 splits][128 rows]
-    static constexpr int SMEM_BYTES = XCHG_OFF + 2 * KS * 128 * 4 + 1024;
+    static constexpr int SMEM_BYTES = MISC_OFF + 256 + 1024;
     static constexpr int O_COLS = D + 16;
     static constexpr bool Q_IN_TMEM = (D == 256);
     static constexpr int QT_COL = 272;                      // d = 256 only
@@ -85,7 +85,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + C::MISC_OFF + 8 * N_BARS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_gen + C::MISC_OFF + 8 * N_BARS + 8);
-    float* xmax = reinterpret_cast<float*>(smem_gen + C::XCHG_OFF);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int N = args.N;
@@ -110,7 +109,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         }
         mbar_init(bar(BAR_SF), 1); mbar_init(bar(BAR_SFREE), NSW);
         mbar_init(bar(BAR_PF), NSW); mbar_init(bar(BAR_PV), 1); mbar_init(bar(BAR_QT), NSW);
-        for (int i = 0; i < 4; ++i) mbar_init(bar(BAR_X + i), KS);
         fence_barrier_init();
     }
     if (warp == W_MMA) { tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS); tmem_relinquish(); }
@@ -208,7 +206,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         const int r_loc = quarter * 32 + lane;                    // row inside the tile = TMEM lane
         const int row = q0 + r_loc;
         const uint32_t t_lane = tmem + ((uint32_t)(quarter * 32) << 16);
-        const uint32_t xbar = bar(BAR_X + quarter);
         const float LOG2E = 1.4426950408889634f;
         const int key_lim = args.causal ? min(row, N - 1) : N - 1;
         int dbg_slot = -1;

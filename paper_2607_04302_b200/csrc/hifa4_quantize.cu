@@ -51,7 +51,7 @@ __device__ __forceinline__ uint32_t quantize8(float (&x)[8], int j, uint32_t (&w
     const int k0 = max(n0, a), k1 = max(n1, a);
     uint32_t part = ((uint32_t)a << (8 + j)) | ((uint32_t)((k0 - a) | ((k1 - a) << 1)) << (16 + 2 * j));
     if (j == 0) part |= (uint32_t)code;
-    uint32_t nib = 0;
+    uint32_t xw[2];                                               // per subgroup: nibbles n0 | n1 << 4 in byte 0, n2 | n3 << 4 in byte 2
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const uint32_t ks = (uint32_t)(h ? k1 : k0) << 23;
@@ -67,12 +67,18 @@ __device__ __forceinline__ uint32_t quantize8(float (&x)[8], int j, uint32_t (&w
         asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[2 * h + 1]) : "f"(v3), "f"(v2));
         unpack2(y01, y[0], y[1]);
         unpack2(y23, y[2], y[3]);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int m = (int)(__float_as_uint(y[i]) - magic_bits);          // signed code
-            nib |= ((uint32_t)abs(m) | ((uint32_t)(m >> 28) & 8u)) << (4 * (4 * h + i));
-        }
+        // The low byte of bits(y) is the signed code m (the magic constant's low byte is 0): gather the
+        // four bytes and turn them into sign-magnitude nibbles with byte-parallel arithmetic.
+        const uint32_t b01 = __byte_perm(__float_as_uint(y[0]), __float_as_uint(y[1]), 0x0040);
+        const uint32_t b23 = __byte_perm(__float_as_uint(y[2]), __float_as_uint(y[3]), 0x0040);
+        const uint32_t bb = __byte_perm(b01, b23, 0x5410);                     // m0, m1, m2, m3 as signed bytes
+        const uint32_t sg = bb & 0x80808080u;                                  // sign bits
+        const uint32_t ng = sg >> 7;                                           // 1 in every negative byte
+        const uint32_t ab = (bb ^ (ng * 0xFFu)) + ng;                          // |m| per byte (no carry between bytes: |m| <= 7)
+        const uint32_t nb = ab | (sg >> 4);                                    // sign to bit 3 of the byte
+        xw[h] = nb | (nb >> 4);
     }
+    const uint32_t nib = __byte_perm(xw[0], xw[1], 0x6420);
     part |= __shfl_xor_sync(0xffffffffu, part, 1);
     part |= __shfl_xor_sync(0xffffffffu, part, 2);
     part |= __shfl_xor_sync(0xffffffffu, part, 4);
@@ -119,18 +125,18 @@ struct QuantJob {                     // one launch quantizes Q, K and V (any of
     float *q_mu, *k_sum;              // Q-Mean auxiliary outputs or null
     int Hq, Hkv, N, d;
     unsigned q_blocks, k_blocks;      // CTAs [0, q_blocks) take Q, the next k_blocks K, the rest V
-    unsigned row_blocks_per_head;     // N * d / 8 / ROW_UNITS_PER_CTA
+    unsigned row_blocks_per_head;     // N * d / 8 / (256 * UPT)
     HeadMap qmap;
 };
 
 constexpr int QUANT_THREADS = 256;
-constexpr int ROW_UNITS_PER_THREAD = 2;
-constexpr int ROW_UNITS_PER_CTA = QUANT_THREADS * ROW_UNITS_PER_THREAD;
+// Row units per thread (template parameter UPT): 4 where a head holds a multiple of 1024 units, which
+// keeps 64 bytes of loads in flight per thread (the kernel is latency-bound below that), else 2.
 
-// Q and K: groups along d.  One head is N*d/8 units of 8 channels; a CTA takes 512 consecutive
-// units, thread t the units t and t + 256 (both loads are issued before any arithmetic).  The two
+// Q and K: groups along d.  One head is N*d/8 units of 8 channels; a CTA takes 256 * UPT consecutive
+// units, thread t the units t, t + 256, ... (all loads are issued before any arithmetic).  The two
 // units share their channel offset, hence their Smooth-QK factors.
-template <typename T>
+template <typename T, int UPT>
 __device__ __forceinline__ void quantize_rows_cta(const uint16_t* __restrict__ x, const float* __restrict__ scale,
                                                   int kv_row, long long head, unsigned blk_in_head, int N, int d,
                                                   uint8_t* __restrict__ codes, uint32_t* __restrict__ meta,
@@ -138,12 +144,12 @@ __device__ __forceinline__ void quantize_rows_cta(const uint16_t* __restrict__ x
                                                   float* __restrict__ ksum_out)
 {
     const int upr = d >> 3;                                                   // units per row
-    const unsigned u0 = blk_in_head * ROW_UNITS_PER_CTA + threadIdx.x;        // unit inside the head
+    const unsigned u0 = blk_in_head * (QUANT_THREADS * UPT) + threadIdx.x;    // unit inside the head
     const long long base = head * (long long)N * upr;                         // first unit of the head
     const int c0 = (int)(u0 & (unsigned)(upr - 1)) << 3;
-    uint4 raw[ROW_UNITS_PER_THREAD];
+    uint4 raw[UPT];
 #pragma unroll
-    for (int r = 0; r < ROW_UNITS_PER_THREAD; ++r)
+    for (int r = 0; r < UPT; ++r)
         raw[r] = __ldg(reinterpret_cast<const uint4*>(x) + base + u0 + r * QUANT_THREADS);
     float sv[8];
     if (scale) {
@@ -153,7 +159,7 @@ __device__ __forceinline__ void quantize_rows_cta(const uint16_t* __restrict__ x
         sv[4] = s1.x; sv[5] = s1.y; sv[6] = s1.z; sv[7] = s1.w;
     }
 #pragma unroll
-    for (int r = 0; r < ROW_UNITS_PER_THREAD; ++r) {
+    for (int r = 0; r < UPT; ++r) {
         const unsigned u = u0 + r * QUANT_THREADS;
         const long long t = base + u;
         const uint32_t rw[4] = {raw[r].x, raw[r].y, raw[r].z, raw[r].w};
@@ -162,9 +168,11 @@ __device__ __forceinline__ void quantize_rows_cta(const uint16_t* __restrict__ x
         for (int i = 0; i < 4; ++i) Pair16<T>::unpack(rw[i], v[2 * i], v[2 * i + 1]);
         if (scale) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-                Pair16<T>::unpack(Pair16<T>::round_pack(v[2 * i] * sv[2 * i], v[2 * i + 1] * sv[2 * i + 1]),
-                                  v[2 * i], v[2 * i + 1]);
+            for (int i = 0; i < 4; ++i) {
+                float a, b;
+                unpack2(mul2(pack2(v[2 * i], v[2 * i + 1]), pack2(sv[2 * i], sv[2 * i + 1])), a, b);
+                Pair16<T>::unpack(Pair16<T>::round_pack(a, b), v[2 * i], v[2 * i + 1]);
+            }
         }
         if (mu_out || ksum_out) {
             // Q-Mean auxiliary (Algorithm 1 lines 2 and 6).  A row of d channels sits in d/8 consecutive,
@@ -228,7 +236,7 @@ __device__ __forceinline__ void quantize_tokens_cta(const uint16_t* __restrict__
     }
 }
 
-template <typename T>
+template <typename T, int UPT>
 __global__ void __launch_bounds__(QUANT_THREADS)
 quantize_qkv_kernel(const __grid_constant__ QuantJob job)
 {
@@ -239,10 +247,10 @@ quantize_qkv_kernel(const __grid_constant__ QuantJob job)
         const unsigned head = blk / job.row_blocks_per_head;             // b * H + h
         const unsigned in_head = blk - head * job.row_blocks_per_head;
         if (is_q)
-            quantize_rows_cta<T>(job.q, job.s, job.qmap.kv_of[head % (unsigned)job.Hq], head, in_head, job.N, job.d,
+            quantize_rows_cta<T, UPT>(job.q, job.s, job.qmap.kv_of[head % (unsigned)job.Hq], head, in_head, job.N, job.d,
                                  job.q_codes, job.q_meta, job.q_img, job.q_mu, nullptr);
         else
-            quantize_rows_cta<T>(job.k, job.inv_s, (int)(head % (unsigned)job.Hkv), head, in_head, job.N, job.d,
+            quantize_rows_cta<T, UPT>(job.k, job.inv_s, (int)(head % (unsigned)job.Hkv), head, in_head, job.N, job.d,
                                  job.k_codes, job.k_meta, job.k_img, nullptr, job.k_sum);
     } else {
         blk -= job.q_blocks + job.k_blocks;
@@ -318,7 +326,9 @@ cudaError_t launch_quantize_qkv(int dtype, const hifa4_shape& sh, const HeadMap&
     job.q_img = (uint16_t*)out.q_mma; job.k_img = (uint16_t*)out.k_mma; job.v_img = (uint16_t*)out.v_mma;
     job.q_mu = out.q_mu; job.k_sum = out.k_sum;
     job.Hq = sh.Hq; job.Hkv = sh.Hkv; job.N = sh.N; job.d = sh.d;
-    job.row_blocks_per_head = (unsigned)((long long)sh.N * sh.d / 8 / ROW_UNITS_PER_CTA);
+    const long long head_units = (long long)sh.N * sh.d / 8;
+    const int upt = head_units % (QUANT_THREADS * 4) == 0 ? 4 : 2;
+    job.row_blocks_per_head = (unsigned)(head_units / (QUANT_THREADS * upt));
     job.q_blocks = q ? (unsigned)sh.B * sh.Hq * job.row_blocks_per_head : 0u;
     job.k_blocks = k ? (unsigned)sh.B * sh.Hkv * job.row_blocks_per_head : 0u;
     const unsigned v_blocks = v ? (unsigned)sh.B * sh.Hkv * (sh.N / 64) * (sh.d / 64) : 0u;
@@ -326,10 +336,13 @@ cudaError_t launch_quantize_qkv(int dtype, const hifa4_shape& sh, const HeadMap&
     const unsigned long long total = (unsigned long long)job.q_blocks + job.k_blocks + v_blocks;
     if (total == 0) return cudaSuccess;
     if (total > 0x7FFFFFFFull) return cudaErrorInvalidConfiguration;
-    if (dtype == HIFA4_F16)
-        quantize_qkv_kernel<__half><<<(unsigned)total, QUANT_THREADS, 0, st>>>(job);
-    else
-        quantize_qkv_kernel<__nv_bfloat16><<<(unsigned)total, QUANT_THREADS, 0, st>>>(job);
+    if (dtype == HIFA4_F16) {
+        if (upt == 4) quantize_qkv_kernel<__half, 4><<<(unsigned)total, QUANT_THREADS, 0, st>>>(job);
+        else quantize_qkv_kernel<__half, 2><<<(unsigned)total, QUANT_THREADS, 0, st>>>(job);
+    } else {
+        if (upt == 4) quantize_qkv_kernel<__nv_bfloat16, 4><<<(unsigned)total, QUANT_THREADS, 0, st>>>(job);
+        else quantize_qkv_kernel<__nv_bfloat16, 2><<<(unsigned)total, QUANT_THREADS, 0, st>>>(job);
+    }
     count_launch();
     return cudaGetLastError();
 }
