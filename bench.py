@@ -31,7 +31,7 @@ UNIT = "TFLOP/s"
 NOMINAL = {"fp4": 9000.0, "fp8": 4500.0, "bf16": 2250.0}      # dense TFLOP/s, context only
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture
 # summarised in profiles/attention_fwd_ws_C2.md (bytes per launch; None where not captured)
-NCU_TRAFFIC_BYTES = {"C2-qwen3-8b-4k": 67.14e6}
+NCU_TRAFFIC_BYTES = {("C2-qwen3-8b-4k", 64): 71.78e6, ("C2-qwen3-8b-4k", 128): 67.14e6}
 
 
 def attn_flops(cfg) -> float:
@@ -354,9 +354,15 @@ def main():
     value = whole_job_tflops(cfg, world, args.steps, total_ms)
     attn_avg_ms = sum(attn_ms) / len(attn_ms)
     achieved = fl / (attn_avg_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "attention_fwd_kernel", "achieved": achieved, "peak": peaks["bf16"],
+    if cfg.Bc == 64 and cfg.d in (128, 256):
+        kern = f"attention_fwd_ws64_kernel<{cfg.d}>"
+    elif cfg.Bc == 128 and cfg.d == 128:
+        kern = "attention_fwd_ws_kernel<4>"
+    else:
+        kern = f"attention_fwd_kernel<{cfg.d},{cfg.Bc}>"
+    roofline = {"bound": "tensor", "kernel": kern, "achieved": achieved, "peak": peaks["bf16"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["bf16"],
-                "traffic": NCU_TRAFFIC_BYTES.get(cfg.name if cfg.causal else None),
+                "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, cfg.Bc) if cfg.causal and not args.p_f32 else None),
                 "peak_source": f"{peaks['source']} cuBLAS bf16 burst (the MMA kind issued is kind::f16 on BF16 images)",
                 "avg_launch_ms": attn_avg_ms,
                 "frac_of_nominal": {k_: achieved / v_ for k_, v_ in NOMINAL.items()}}
