@@ -366,6 +366,9 @@ int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv&
         a.dbg.p_codes = dbg->p_codes; a.dbg.p_step = dbg->p_step;
         a.dbg.l_out = dbg->l_out; a.dbg.m_out = dbg->m_out;
     }
+    // Head-major order pays once the K-hat and V-hat^T images of all KV heads exceed L2 (126 MB) well:
+    // measured on B = 4, Hkv = 8, d = 128: slower at N = 8192 (134 MB), +4 % at 16384, +7 % at 32768.
+    a.head_major = (double)sh.B * sh.Hkv * sh.N * sh.d * 4.0 > 200e6 ? 1 : 0;
     a.normalizer = prm.normalizer ? 1 : 0;
     a.p_f32 = prm.p_dtype == HIFA4_F32 ? 1 : 0;
     if (a.p_f32) {                                // variant built for the 64-key warp-specialised kernels only

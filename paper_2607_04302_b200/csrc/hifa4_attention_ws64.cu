@@ -91,8 +91,10 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     const int n_qt = (N + 127) / 128;
     // 1-D grid, query block outermost and descending: the heaviest causal CTAs are scheduled first
     const int n_bh = args.B * args.Hq;
-    const int qt = n_qt - 1 - (int)(blockIdx.x / n_bh);
-    const int bh = (int)(blockIdx.x % n_bh);
+    // Long sequences, whose K/V images do not fit in L2 together: head outermost instead, so that the
+    // CTAs in flight share the K/V of one or two heads; still heaviest first inside a head.
+    const int qt = n_qt - 1 - (int)(args.head_major ? blockIdx.x % n_qt : blockIdx.x / n_bh);
+    const int bh = (int)(args.head_major ? blockIdx.x / n_qt : blockIdx.x % n_bh);
     const int h = bh % args.Hq, b = bh / args.Hq;
     const int g = args.map.kv_of[h];
     const int q0 = qt * 128;

@@ -135,6 +135,15 @@ def test_sweep_point_8k_sampled(hb, par, Bc):
     print(par.assert_within_bars(res, "C5 N=8192 causal"))
 
 
+def test_long_sequence_head_major_order_sampled(hb, par):
+    """B = 4, Hkv = 8, N = 16384: the K/V images (268 MB) exceed L2, so the 64-key kernel launches its CTAs
+    head by head instead of query block by query block; sampled rows against the oracle."""
+    cfg = synth.config("C5", N=16384, Hq=8, Hkv=8, cal_samples=2, cal_tokens=256)
+    blocks = [(0, 0, 0), (3, 7, 127), (1, 3, 64), (2, 5, 1)]
+    res = par.run_case(cfg, DEV, blocks=blocks, check_quant=False, rows_per_block=6)
+    print(par.assert_within_bars(res, "C5-like N=16384 head-major"))
+
+
 @pytest.mark.parametrize("causal,Bc", [(True, 64), (False, 64), (True, 128)])
 def test_largest_sequence_properties(hb, causal, Bc):
     """N = 32768 (the top of the sequence sweep), too large for the oracle: properties that hold at any
