@@ -389,7 +389,7 @@ int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv&
         if (sh.d == 256 && prm.Bc == 64) return launch_cfg<256, 64, true>(sh, qkv, a, st);
         return HIFA4_ERR_UNSUPPORTED;
     }
-    if (sh.d == 64 && prm.Bc == 64) return launch_cfg<64, 64, false>(sh, qkv, a, st);
+    if (sh.d == 64 && prm.Bc == 64) return launch_attention_ws64(sh, qkv, a, st);
     if (sh.d == 64 && prm.Bc == 128) return launch_cfg<64, 128, false>(sh, qkv, a, st);
     if (sh.d == 128 && prm.Bc == 64) return launch_attention_ws64(sh, qkv, a, st);
     if (sh.d == 128 && prm.Bc == 128) return launch_attention_ws(sh, qkv, a, st);

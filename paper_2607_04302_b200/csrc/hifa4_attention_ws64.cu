@@ -1,4 +1,4 @@
-// Warp-specialised HiFA4 attention forward for Bc = 64 (Algorithm 1 lines 4-13), d = 128 or 256.
+// Warp-specialised HiFA4 attention forward for Bc = 64 (Algorithm 1 lines 4-13), d = 64, 128 or 256.
 //
 // One CTA = 128 query rows of one (batch, query head), 10 warps:
 //   warps 0-7  softmax / quantize: warp w owns rows 32*(w%4).. of the tile and keys 32*(w/4).. of
@@ -13,6 +13,7 @@
 //   d = 256: 512 tensor-memory columns: [O | l] 0..271 (an N = 256 MMA for the channels, an N = 16
 //            MMA on the same A operand for the ones block), Q-hat image 272..399 (A operand of
 //            Q K^T from tensor memory), S 400..463, P-hat 464..495.  One CTA per SM.
+//   d = 64:  as d = 128 with [O | l] 0..79 (one N = 80 MMA); 53 KB of shared memory.
 //   d = 128: 256 tensor-memory columns: [O | l] 0..143 (one N = 144 MMA), S 144..207, P-hat
 //            208..239; Q-hat stays in shared memory (SS-form Q K^T).  101 KB of shared memory and
 //            <= 102 registers, so two CTAs share an SM and fill each other's synchronisation gaps.
@@ -550,6 +551,7 @@ int launch_attention_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const Att
     }
     if (sh.d == 256) return dbg ? launch_ws64<256, true, false>(sh, qkv, args, st) : launch_ws64<256, false, false>(sh, qkv, args, st);
     if (sh.d == 128) return dbg ? launch_ws64<128, true, false>(sh, qkv, args, st) : launch_ws64<128, false, false>(sh, qkv, args, st);
+    if (sh.d == 64) return dbg ? launch_ws64<64, true, false>(sh, qkv, args, st) : launch_ws64<64, false, false>(sh, qkv, args, st);
     return HIFA4_ERR_UNSUPPORTED;
 }
 

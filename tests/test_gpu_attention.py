@@ -43,6 +43,7 @@ SMALL = {
     "d128-bc64-noncausal": synth.config("C3", N=192, Hq=1, Hkv=1, causal=False),
     "d64-bc128": synth.config("C3", N=256, Hq=2, Hkv=1, d=64, Bc=128),
     "d64-bc64-fp16": synth.config("C3", N=256, Hq=2, Hkv=1, d=64, Bc=64, dtype="fp16"),
+    "d64-bc64-causal-gqa-ragged": synth.config("C2", N=448, Hq=4, Hkv=2, d=64, cal_samples=3, cal_tokens=64),
     "d256-bc64-mild": synth.config("C4", N=256, Hq=2, Hkv=1, Bc=64, cal_samples=3, cal_tokens=64),
     "batch2": synth.config("C5", B=2, N=256, Hq=4, Hkv=2, Bc=128, cal_samples=2, cal_tokens=64),
     "batch2-bc64": synth.config("C5", B=2, N=256, Hq=4, Hkv=2, cal_samples=2, cal_tokens=64),
