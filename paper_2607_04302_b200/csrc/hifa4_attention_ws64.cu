@@ -76,7 +76,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     constexpr int W_TMA = C::W_TMA, W_MMA = C::W_MMA, KPT = C::KPT, NU = C::NU, QSUB = C::QSUB;
     constexpr int Q_BYTES = C::Q_BYTES, K_SUB = C::K_SUB, K_STAGE = C::K_STAGE, V_STAGE = C::V_STAGE;
     constexpr int O_COLS = C::O_COLS, QT_COL = C::QT_COL, S_COL = C::S_COL, P_COL = C::P_COL, TMEM_COLS = C::TMEM_COLS;
-    if (args.d_status && *reinterpret_cast<volatile int*>(args.d_status) != 0) return;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -123,16 +122,24 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     }
     fence_proxy_async_smem();
     tc_fence_before();
+    // The launch lets this grid start while its predecessor in the stream is still running (its CTAs
+    // become resident and set themselves up as SMs drain); nothing the predecessor wrote is touched
+    // before this point.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // a CTA that starts after another one reported a failure does nothing
+    const bool dead = args.d_status && *reinterpret_cast<volatile int*>(args.d_status) != 0;
 
     auto fail = [&](int site) {
         *abort_flag = 1;
         if (args.d_status) atomicCAS(args.d_status, 0, HIFA4_ERR_TIMEOUT + 16 * site);
     };
 
-    if (warp == W_TMA) {
+    if (dead) {
+        // fall through to the common exit
+    } else if (warp == W_TMA) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             mbar_expect_tx(bar(BAR_Q), Q_BYTES);
@@ -536,9 +543,19 @@ static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnAr
         attr_set = true;
     }
     dim3 grid((unsigned)(((sh.N + 127) / 128) * sh.Hq * sh.B));
-    kern<<<grid, C::THREADS, C::SMEM_BYTES, st>>>(mq, mk, mv, args);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(C::THREADS);
+    cfg.dynamicSmemBytes = C::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see griddepcontrol.wait in the kernel
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, mq, mk, mv, args);
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? HIFA4_OK : HIFA4_ERR_CUDA;
+    return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? HIFA4_OK : HIFA4_ERR_CUDA;
 }
 
 int launch_attention_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)

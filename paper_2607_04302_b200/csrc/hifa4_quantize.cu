@@ -240,6 +240,9 @@ template <typename T, int UPT>
 __global__ void __launch_bounds__(QUANT_THREADS)
 quantize_qkv_kernel(const __grid_constant__ QuantJob job)
 {
+    // a dependent grid launched with programmatic stream serialization (the attention kernel) may start
+    // becoming resident as this grid's CTAs retire; it waits for this grid's completion before it reads
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     unsigned blk = blockIdx.x;
     if (blk < job.q_blocks + job.k_blocks) {
         const bool is_q = blk < job.q_blocks;
