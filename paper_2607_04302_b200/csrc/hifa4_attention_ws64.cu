@@ -25,9 +25,12 @@ namespace hifa4 {
 #ifndef HIFA4_WS64_KS128
 #define HIFA4_WS64_KS128 2
 #endif
+#ifndef HIFA4_WS64_KS256
+#define HIFA4_WS64_KS256 2
+#endif
 template <int D_>
 struct WS64 {
-    static constexpr int D = D_, BC = 64, STAGES = 2, KS = (D_ == 128) ? HIFA4_WS64_KS128 : 2;
+    static constexpr int D = D_, BC = 64, STAGES = 2, KS = (D_ == 128) ? HIFA4_WS64_KS128 : (D_ == 256 ? HIFA4_WS64_KS256 : 2);
     static constexpr int NSW = 4 * KS, THREADS = (NSW + 2) * 32, W_TMA = NSW, W_MMA = NSW + 1;
     static constexpr int KPT = BC / KS, NU = KPT / 8;       // 32 keys = 4 level-2 units per thread and tile
     static constexpr int QSUB = D / 64;                     // 64-channel sub-tiles of Q and K
@@ -231,20 +234,21 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         // channels of its row = 64 columns of packed BF16 pairs.  (d = 128: the issuer waits for the
         // Q load itself.)
         if constexpr (C::Q_IN_TMEM) {
-            static_assert(!C::Q_IN_TMEM || KS == 2, "the Q copy splits a row over two threads");
+            static_assert(!C::Q_IN_TMEM || KS == 2 || KS == 4, "the Q copy splits a row over two or four threads");
             if (wait64(bar(BAR_Q), 0, abort_flag)) {
                 const int sw = r_loc & 7;
+                constexpr int PARTS = 4 / KS;                          // pieces of 64 channels (8 chunks, 32 columns)
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
+                for (int half = 0; half < PARTS; ++half) {
                     uint32_t qw[32];
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
-                        const int chunk = kq * 16 + half * 8 + c;      // 16-byte chunk of the 512-byte row
+                        const int chunk = (kq * PARTS + half) * 8 + c; // 16-byte chunk of the 512-byte row
                         const uint32_t a = q_s + (chunk >> 3) * 16384 + (r_loc >> 3) * 1024 + sw * 128 + (((chunk & 7) ^ sw) << 4);
                         asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                                      : "=r"(qw[4 * c]), "=r"(qw[4 * c + 1]), "=r"(qw[4 * c + 2]), "=r"(qw[4 * c + 3]) : "r"(a));
                     }
-                    tmem_st32(t_lane + QT_COL + kq * 64 + half * 32, qw);
+                    tmem_st32(t_lane + QT_COL + (kq * PARTS + half) * 32, qw);
                 }
                 tmem_wait_st();
                 tc_fence_before();
@@ -274,10 +278,16 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                     tmem_wait_ld();
 #pragma unroll
                     for (int i = 0; i < 32; ++i) r[32 + i] = r1[i];
-                } else {
-                    static_assert(KS <= 2, "key split of one or two threads per row");
+                } else if constexpr (KS == 2) {
                     tmem_ld32(t_lane + S_COL + kq * KPT, reinterpret_cast<uint32_t(&)[32]>(r[0]));
                     tmem_ld32(t_lane + S_COL + (kq ^ 1) * KPT, reinterpret_cast<uint32_t(&)[32]>(ro[0]));
+                    tmem_wait_ld();
+                } else {
+                    static_assert(KS == 4, "key split of one, two or four threads per row");
+                    tmem_ld16(t_lane + S_COL + kq * KPT, reinterpret_cast<uint32_t(&)[16]>(r[0]));
+#pragma unroll
+                    for (int o = 1; o < KS; ++o)               // part kq ^ o of the row goes to ro[(o - 1) * KPT ..]
+                        tmem_ld16(t_lane + S_COL + (kq ^ o) * KPT, reinterpret_cast<uint32_t(&)[16]>(ro[(o - 1) * KPT]));
                     tmem_wait_ld();
                 }
 #pragma unroll
@@ -289,7 +299,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(BAR_SFREE));
 
-            const int obase = j0 + (kq ^ 1) * KPT;             // first key of the other part of the row (KS = 2)
+            auto obase = [&](int o) { return j0 + (kq ^ o) * KPT; };   // first key of the o-th other part of the row
             if (args.qmean) {                                  // Q-Mean correction (line 6): + mu_i * sum_c k~_jc
                 if (kbase < N) {
                     const float4* kp = reinterpret_cast<const float4*>(args.k_sum + (size_t)bh_kv * N + kbase);
@@ -302,15 +312,19 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                         p[4 * i + 3] = fmaf(mu_row, ks.w, p[4 * i + 3]);
                     }
                 }
-                if (KS > 1 && obase < N) {
-                    const float4* kp = reinterpret_cast<const float4*>(args.k_sum + (size_t)bh_kv * N + obase);
 #pragma unroll
-                    for (int i = 0; i < (BC - KPT) / 4; ++i) {
-                        const float4 ks = __ldg(kp + i);
-                        po[4 * i] = fmaf(mu_row, ks.x, po[4 * i]);
-                        po[4 * i + 1] = fmaf(mu_row, ks.y, po[4 * i + 1]);
-                        po[4 * i + 2] = fmaf(mu_row, ks.z, po[4 * i + 2]);
-                        po[4 * i + 3] = fmaf(mu_row, ks.w, po[4 * i + 3]);
+                for (int o = 1; o < KS; ++o) {
+                    if (obase(o) < N) {
+                        const float4* kp = reinterpret_cast<const float4*>(args.k_sum + (size_t)bh_kv * N + obase(o));
+                        float* q4 = po + (o - 1) * KPT;
+#pragma unroll
+                        for (int i = 0; i < KPT / 4; ++i) {
+                            const float4 ks = __ldg(kp + i);
+                            q4[4 * i] = fmaf(mu_row, ks.x, q4[4 * i]);
+                            q4[4 * i + 1] = fmaf(mu_row, ks.y, q4[4 * i + 1]);
+                            q4[4 * i + 2] = fmaf(mu_row, ks.z, q4[4 * i + 2]);
+                            q4[4 * i + 3] = fmaf(mu_row, ks.w, q4[4 * i + 3]);
+                        }
                     }
                 }
             }
@@ -319,7 +333,10 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
 #pragma unroll
                 for (int i = 0; i < KPT; ++i) p[i] = (kbase + i > key_lim) ? -INFINITY : p[i];
 #pragma unroll
-                for (int i = 0; i < BC - KPT; ++i) po[i] = (obase + i > key_lim) ? -INFINITY : po[i];
+                for (int o = 1; o < KS; ++o)
+#pragma unroll
+                    for (int i = 0; i < KPT; ++i)
+                        po[(o - 1) * KPT + i] = (obase(o) + i > key_lim) ? -INFINITY : po[(o - 1) * KPT + i];
             }
             float mx;
             {
@@ -328,8 +345,10 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 for (int i = 0; i < KPT / 4; ++i) t4[i] = fmaxf(max3(p[4 * i], p[4 * i + 1], p[4 * i + 2]), p[4 * i + 3]);
                 if constexpr (KS > 1) {
 #pragma unroll
-                    for (int i = 0; i < (BC - KPT) / 4; ++i)
-                        t4[i] = fmaxf(max3(t4[i], po[4 * i], po[4 * i + 1]), fmaxf(po[4 * i + 2], po[4 * i + 3]));
+                    for (int i = 0; i < (BC - KPT) / 4; ++i) {
+                        float& t = t4[i % (KPT / 4)];
+                        t = fmaxf(max3(t, po[4 * i], po[4 * i + 1]), fmaxf(po[4 * i + 2], po[4 * i + 3]));
+                    }
                 }
 #pragma unroll
                 for (int w = KPT / 8; w >= 1; w >>= 1)
