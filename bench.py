@@ -203,6 +203,7 @@ def main():
     ap.add_argument("--Bc", type=int, default=0, help="key-tile width (default: the configuration's, 64)")
     ap.add_argument("--p-f32", action="store_true",
                     help="variant: quantize the FP32 exponential (not the method's FP16 P; for comparison only)")
+    ap.add_argument("--qmean", action="store_true", help="with the Q-Mean auxiliary (Algorithm 1 lines 2 and 6)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -250,7 +251,7 @@ def main():
         qc, kc = synth.make_calibration(cfg, samples=min(cfg.cal_samples, 8), tokens=min(cfg.cal_tokens, 512))
         s, inv_s = hb.smooth_calibrate(qc.to(dev), kc.to(dev), cfg.smooth_mode)
     dt = hb._DT[q.dtype]
-    qkv = hb.alloc_qkv(cfg.B, cfg.Hq, cfg.Hkv, cfg.N, cfg.d, dt, dev)
+    qkv = hb.alloc_qkv(cfg.B, cfg.Hq, cfg.Hkv, cfg.N, cfg.d, dt, dev, qmean=args.qmean)
     out = torch.empty((cfg.B, cfg.Hq, cfg.N, cfg.d), dtype=torch.float32, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)       # > 126 MB of L2
@@ -267,13 +268,13 @@ def main():
         """One pass of the hot path.  split: record an event between the two launches (used only by the
         pass that attributes time to each kernel: the event keeps the attention grid, which is launched
         with programmatic stream serialization, from starting while the quantize grid drains)."""
-        hb.quantize_qkv(q, k, v, s, inv_s, out=qkv, d_status=status)
+        hb.quantize_qkv(q, k, v, s, inv_s, out=qkv, d_status=status, qmean=args.qmean)
         mid = None
         if split:
             mid = torch.cuda.Event(enable_timing=True)
             mid.record()
         hb.attention_fwd(qkv, cfg.causal, Bc=cfg.Bc, out_dtype=hb.F32, out=out, d_status=status,
-                         p_dtype=hb.F32 if args.p_f32 else hb.F16)
+                         p_dtype=hb.F32 if args.p_f32 else hb.F16, qmean=args.qmean)
         return mid
 
     def barrier():
@@ -333,7 +334,7 @@ def main():
 
     # ---- end to end through the raw C-ABI entry point with host buffers (pinned), copies timed
     e2e = None
-    if not big:
+    if not big and not args.qmean:
         pq, pk, pv = qh.pin_memory(), kh.pin_memory(), vh.pin_memory()
         po = torch.empty(out.shape, dtype=torch.float32).pin_memory()
         dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
@@ -444,7 +445,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "N": cfg.N, "d": cfg.d,
                        "causal": cfg.causal, "Br": 128, "Bc": cfg.Bc, "in_dtype": cfg.dtype, "out_dtype": "f32",
-                       "p_dtype": "f32 (variant)" if args.p_f32 else "f16",
+                       "p_dtype": "f32 (variant)" if args.p_f32 else "f16", "qmean": bool(args.qmean),
                        "smooth_mode": cfg.smooth_mode, "step": "hifa4_quantize_qkv + hifa4_attention_fwd",
                        "l2": "flushed between steps (256 MiB write, then a 256 MiB read that drains the dirty lines), outside the per-step events",
                        "parallelism": f"replicated batches x{world}"},

@@ -42,7 +42,8 @@ struct WS64 {
     static constexpr int K_OFF = Q_OFF + Q_BYTES;
     static constexpr int V_OFF = K_OFF + STAGES * K_STAGE;
     static constexpr int MISC_OFF = V_OFF + STAGES * V_STAGE;
-    static constexpr int SMEM_BYTES = MISC_OFF + 256 + 1024;
+    static constexpr int KSUM_OFF = MISC_OFF + 256;         // Q-Mean: channel sums of the tile's 64 keys, two stages
+    static constexpr int SMEM_BYTES = KSUM_OFF + STAGES * 256 + 1024;
     static constexpr int O_COLS = D + 16;
     static constexpr bool Q_IN_TMEM = (D == 256);
     static constexpr int QT_COL = 272;                      // d = 256 only
@@ -53,7 +54,7 @@ struct WS64 {
 };
 namespace ws64 {
 enum { BAR_Q = 0, BAR_KF = 1, BAR_KE = 3, BAR_VF = 5, BAR_VE = 7, BAR_SF = 9, BAR_SFREE = 10, BAR_PF = 11,
-       BAR_PV = 12, BAR_X = 13, BAR_QT = 17, N_BARS = 18 };
+       BAR_PV = 12, BAR_KSF = 13, BAR_QT = 17, N_BARS = 18 };
 constexpr uint32_t WAIT_POLLS = 1u << 20;
 }  // namespace ws64
 
@@ -114,6 +115,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         }
         mbar_init(bar(BAR_SF), 1); mbar_init(bar(BAR_SFREE), NSW);
         mbar_init(bar(BAR_PF), NSW); mbar_init(bar(BAR_PV), 1); mbar_init(bar(BAR_QT), NSW);
+        mbar_init(bar(BAR_KSF), 1); mbar_init(bar(BAR_KSF + 1), 1);
         fence_barrier_init();
     }
     if (warp == W_MMA) { tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS); tmem_relinquish(); }
@@ -160,6 +162,12 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 if (!wait64(bar(BAR_VE + st), ph ^ 1u, abort_flag)) { fail(2); break; }
                 mbar_expect_tx(bar(BAR_VF + st), D * 128);
                 tma_load_3d(v_s + st * V_STAGE, &tmap_v, bar(BAR_VF + st), j0, 0, bh_kv);
+                if (args.qmean) {
+                    // Q-Mean: the 64 channel sums of this tile's keys; their stage is free with the V stage
+                    // (PV(jt-2) complete means every softmax warp is past tile jt-2)
+                    mbar_expect_tx(bar(BAR_KSF + st), 256);
+                    bulk_load(smem_base + C::KSUM_OFF + st * 256, args.k_sum + (size_t)bh_kv * N + j0, 256, bar(BAR_KSF + st));
+                }
             }
         }
     } else if (warp == W_MMA) {
@@ -301,32 +309,23 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
 
             auto obase = [&](int o) { return j0 + (kq ^ o) * KPT; };   // first key of the o-th other part of the row
             if (args.qmean) {                                  // Q-Mean correction (line 6): + mu_i * sum_c k~_jc
-                if (kbase < N) {
-                    const float4* kp = reinterpret_cast<const float4*>(args.k_sum + (size_t)bh_kv * N + kbase);
+                if (!wait64(bar(BAR_KSF + (jt & 1)), (uint32_t)(jt >> 1) & 1u, abort_flag)) { fail(15); ok = false; break; }
+                const uint32_t ks_s = smem_base + C::KSUM_OFF + (jt & 1) * 256;
+                auto add_part = [&](float* dst, int part) {     // keys part * KPT .. of the tile
 #pragma unroll
                     for (int i = 0; i < KPT / 4; ++i) {
-                        const float4 ks = __ldg(kp + i);
-                        p[4 * i] = fmaf(mu_row, ks.x, p[4 * i]);
-                        p[4 * i + 1] = fmaf(mu_row, ks.y, p[4 * i + 1]);
-                        p[4 * i + 2] = fmaf(mu_row, ks.z, p[4 * i + 2]);
-                        p[4 * i + 3] = fmaf(mu_row, ks.w, p[4 * i + 3]);
+                        float4 ks;
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                     : "=f"(ks.x), "=f"(ks.y), "=f"(ks.z), "=f"(ks.w) : "r"(ks_s + (part * KPT + 4 * i) * 4));
+                        dst[4 * i] = fmaf(mu_row, ks.x, dst[4 * i]);
+                        dst[4 * i + 1] = fmaf(mu_row, ks.y, dst[4 * i + 1]);
+                        dst[4 * i + 2] = fmaf(mu_row, ks.z, dst[4 * i + 2]);
+                        dst[4 * i + 3] = fmaf(mu_row, ks.w, dst[4 * i + 3]);
                     }
-                }
+                };
+                add_part(p, kq);
 #pragma unroll
-                for (int o = 1; o < KS; ++o) {
-                    if (obase(o) < N) {
-                        const float4* kp = reinterpret_cast<const float4*>(args.k_sum + (size_t)bh_kv * N + obase(o));
-                        float* q4 = po + (o - 1) * KPT;
-#pragma unroll
-                        for (int i = 0; i < KPT / 4; ++i) {
-                            const float4 ks = __ldg(kp + i);
-                            q4[4 * i] = fmaf(mu_row, ks.x, q4[4 * i]);
-                            q4[4 * i + 1] = fmaf(mu_row, ks.y, q4[4 * i + 1]);
-                            q4[4 * i + 2] = fmaf(mu_row, ks.z, q4[4 * i + 2]);
-                            q4[4 * i + 3] = fmaf(mu_row, ks.w, q4[4 * i + 3]);
-                        }
-                    }
-                }
+                for (int o = 1; o < KS; ++o) add_part(po + (o - 1) * KPT, kq ^ o);
             }
             const bool need_mask = (args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N);
             if (need_mask) {                                   // masked scores become -inf: exp gives exact zeros
