@@ -69,7 +69,7 @@ static __device__ __forceinline__ bool wait64(uint32_t bar, uint32_t parity, vol
     return false;
 }
 
-template <int DH, bool DBG, bool PF32>
+template <int DH, bool DBG, bool PF32, bool QM>
 __global__ void __launch_bounds__(WS64<DH>::THREADS, WS64<DH>::CTAS_PER_SM)
 attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                            const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnArgs args)
@@ -107,7 +107,10 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     const int n_tiles = last_key / BC + 1;
 
     if (tid == 0) {
-        *abort_flag = 0;
+        // A CTA that starts after another one reported a failure does nothing.  One thread reads the status
+        // word (the load is in flight during the set-up below) and publishes the verdict through shared
+        // memory, so that all roles of the CTA agree on it.
+        const int status_now = args.d_status ? *reinterpret_cast<volatile int*>(args.d_status) : 0;
         mbar_init(bar(BAR_Q), 1);
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar(BAR_KF + s), 1); mbar_init(bar(BAR_KE + s), 1);
@@ -117,6 +120,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         mbar_init(bar(BAR_PF), NSW); mbar_init(bar(BAR_PV), 1); mbar_init(bar(BAR_QT), NSW);
         mbar_init(bar(BAR_KSF), 1); mbar_init(bar(BAR_KSF + 1), 1);
         fence_barrier_init();
+        *abort_flag = status_now != 0 ? 2 : 0;
     }
     if (warp == W_MMA) { tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS); tmem_relinquish(); }
     if (warp == W_TMA && lane == 0) { tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_k); tma_prefetch_desc(&tmap_v); }
@@ -134,8 +138,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    // a CTA that starts after another one reported a failure does nothing
-    const bool dead = args.d_status && *reinterpret_cast<volatile int*>(args.d_status) != 0;
+    const bool dead = *abort_flag != 0;
 
     auto fail = [&](int site) {
         *abort_flag = 1;
@@ -162,7 +165,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 if (!wait64(bar(BAR_VE + st), ph ^ 1u, abort_flag)) { fail(2); break; }
                 mbar_expect_tx(bar(BAR_VF + st), D * 128);
                 tma_load_3d(v_s + st * V_STAGE, &tmap_v, bar(BAR_VF + st), j0, 0, bh_kv);
-                if (args.qmean) {
+                if (QM) {
                     // Q-Mean: the 64 channel sums of this tile's keys; their stage is free with the V stage
                     // (PV(jt-2) complete means every softmax warp is past tile jt-2)
                     mbar_expect_tx(bar(BAR_KSF + st), 256);
@@ -234,7 +237,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             for (int i = 0; i < args.dbg.n_blocks; ++i)
                 if (args.dbg.blocks[3 * i] == b && args.dbg.blocks[3 * i + 1] == h && args.dbg.blocks[3 * i + 2] == qt)
                     dbg_slot = i;
-        const float mu_row = (args.qmean && row < N) ? args.q_mu[(size_t)bh_q * N + row] : 0.f;
+        const float mu_row = (QM && row < N) ? args.q_mu[(size_t)bh_q * N + row] : 0.f;
         float m_run = -INFINITY;
         bool ok = true;
 
@@ -308,7 +311,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             if (lane == 0) mbar_arrive(bar(BAR_SFREE));
 
             auto obase = [&](int o) { return j0 + (kq ^ o) * KPT; };   // first key of the o-th other part of the row
-            if (args.qmean) {                                  // Q-Mean correction (line 6): + mu_i * sum_c k~_jc
+            if (QM) {                                          // Q-Mean correction (line 6): + mu_i * sum_c k~_jc
                 if (!wait64(bar(BAR_KSF + (jt & 1)), (uint32_t)(jt >> 1) & 1u, abort_flag)) { fail(15); ok = false; break; }
                 const uint32_t ks_s = smem_base + C::KSUM_OFF + (jt & 1) * 256;
                 auto add_part = [&](float* dst, int part) {     // keys part * KPT .. of the tile
@@ -545,7 +548,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     if (warp == W_MMA) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
 }
 
-template <int DH, bool DBG, bool PF32>
+template <int DH, bool DBG, bool PF32, bool QM>
 static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
     using C = WS64<DH>;
@@ -553,7 +556,7 @@ static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnAr
     if (!make_bf16_map(&mq, qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, DH, 128)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, DH, C::BC)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, DH, sh.N, DH)) return HIFA4_ERR_CUDA;
-    auto kern = attention_fwd_ws64_kernel<DH, DBG, PF32>;
+    auto kern = attention_fwd_ws64_kernel<DH, DBG, PF32, QM>;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
@@ -576,17 +579,27 @@ static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnAr
     return e == cudaSuccess && cudaGetLastError() == cudaSuccess ? HIFA4_OK : HIFA4_ERR_CUDA;
 }
 
-int launch_attention_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
+template <int DH>
+static int launch_ws64_d(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
     const bool dbg = args.dbg.n_blocks > 0;
-    if (args.p_f32) {
-        if (sh.d == 256) return dbg ? launch_ws64<256, true, true>(sh, qkv, args, st) : launch_ws64<256, false, true>(sh, qkv, args, st);
-        if (sh.d == 128) return dbg ? launch_ws64<128, true, true>(sh, qkv, args, st) : launch_ws64<128, false, true>(sh, qkv, args, st);
-        return HIFA4_ERR_UNSUPPORTED;
+    if (args.p_f32) {                                      // variant: no Q-Mean, d = 128 or 256
+        if constexpr (DH == 64) return HIFA4_ERR_UNSUPPORTED;
+        else {
+            if (args.qmean) return HIFA4_ERR_UNSUPPORTED;
+            return dbg ? launch_ws64<DH, true, true, false>(sh, qkv, args, st) : launch_ws64<DH, false, true, false>(sh, qkv, args, st);
+        }
     }
-    if (sh.d == 256) return dbg ? launch_ws64<256, true, false>(sh, qkv, args, st) : launch_ws64<256, false, false>(sh, qkv, args, st);
-    if (sh.d == 128) return dbg ? launch_ws64<128, true, false>(sh, qkv, args, st) : launch_ws64<128, false, false>(sh, qkv, args, st);
-    if (sh.d == 64) return dbg ? launch_ws64<64, true, false>(sh, qkv, args, st) : launch_ws64<64, false, false>(sh, qkv, args, st);
+    if (args.qmean)
+        return dbg ? launch_ws64<DH, true, false, true>(sh, qkv, args, st) : launch_ws64<DH, false, false, true>(sh, qkv, args, st);
+    return dbg ? launch_ws64<DH, true, false, false>(sh, qkv, args, st) : launch_ws64<DH, false, false, false>(sh, qkv, args, st);
+}
+
+int launch_attention_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
+{
+    if (sh.d == 256) return launch_ws64_d<256>(sh, qkv, args, st);
+    if (sh.d == 128) return launch_ws64_d<128>(sh, qkv, args, st);
+    if (sh.d == 64) return launch_ws64_d<64>(sh, qkv, args, st);
     return HIFA4_ERR_UNSUPPORTED;
 }
 
