@@ -31,7 +31,7 @@ UNIT = "TFLOP/s"
 NOMINAL = {"fp4": 9000.0, "fp8": 4500.0, "bf16": 2250.0}      # dense TFLOP/s, context only
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture
 # summarised in profiles/attention_fwd_ws_C2.md (bytes per launch; None where not captured)
-NCU_TRAFFIC_BYTES = {("C2-qwen3-8b-4k", 64): 71.78e6, ("C2-qwen3-8b-4k", 128): 67.14e6}
+NCU_TRAFFIC_BYTES = {("C2-qwen3-8b-4k", 64): 68.70e6, ("C2-qwen3-8b-4k", 128): 67.14e6}
 
 
 def attn_flops(cfg) -> float:
