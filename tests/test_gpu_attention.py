@@ -206,3 +206,18 @@ def test_qmean_full_size_sampled(hb, par):
     blocks = [(0, 0, 0), (3, 31, 31), (1, 12, 17)]
     res = par.run_case(cfg, DEV, blocks=blocks, check_quant=False, rows_per_block=16, qkv_host=(q, k, v), qmean=True)
     print(par.assert_within_bars(res, "C5 N=4096 qmean"))
+
+
+def test_uneven_head_map_equals_reordered_heads(hb, par):
+    """An explicit query-head -> KV-head map with groups of different sizes and interleaved members gives,
+    head by head, what the default grouping gives on the correspondingly gathered K/V heads."""
+    cfg = synth.config("C3", N=320, Hq=4, Hkv=2)
+    q, k, v = (t.to(DEV) for t in synth.make_qkv(cfg))
+    head_map = [1, 0, 1, 1]                                     # three heads on KV head 1, one on KV head 0
+    mapped = hb.attention_fwd(hb.quantize_qkv(q, k, v, q_to_kv=head_map), True, Bc=64)
+    idx = torch.tensor(head_map, device=DEV)
+    mha = hb.attention_fwd(hb.quantize_qkv(q, k[:, idx].contiguous(), v[:, idx].contiguous()), True, Bc=64)
+    assert torch.equal(mapped, mha)
+    mapped128 = hb.attention_fwd(hb.quantize_qkv(q, k, v, q_to_kv=head_map), True, Bc=128)
+    mha128 = hb.attention_fwd(hb.quantize_qkv(q, k[:, idx].contiguous(), v[:, idx].contiguous()), True, Bc=128)
+    assert torch.equal(mapped128, mha128)
