@@ -206,6 +206,7 @@ def main():
     ap.add_argument("--qmean", action="store_true", help="with the Q-Mean auxiliary (Algorithm 1 lines 2 and 6)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-context", action="store_true", help="skip the torch SDPA / N=8192 context numbers")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -397,6 +398,50 @@ def main():
                "how": f"hifa4_attention_fwd_raw per (batch, KV head group) slice, {len(slices)} slices over "
                       f"{len(streams)} streams, pinned host buffers"}
 
+    # ---- context (not the product): torch SDPA in BF16 on the same inputs, and, for the headline
+    # workload, its N = 8192 sibling (the target sentence names an 8K prefill, the configuration 4K)
+    context = {}
+    if rank == 0 and not args.no_context:
+        import torch.nn.functional as F
+        try:
+            qb, kb, vb = (t.to(torch.bfloat16) for t in (q, k, v))
+            for _ in range(3):
+                F.scaled_dot_product_attention(qb, kb, vb, is_causal=cfg.causal, enable_gqa=True)
+            torch.cuda.synchronize()
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(10):
+                F.scaled_dot_product_attention(qb, kb, vb, is_causal=cfg.causal, enable_gqa=True)
+            b.record()
+            torch.cuda.synchronize()
+            context["torch_sdpa_bf16_tflops"] = attn_flops(cfg) * 10 / (a.elapsed_time(b) * 1e-3) / 1e12
+        except Exception as e:                                         # context only: never fail the bench on it
+            context["torch_sdpa_bf16_tflops"] = None
+            context["torch_sdpa_error"] = str(e)[:120]
+        if cfg.name == synth.CONFIGS["C2"].name and cfg.N == 4096:
+            c8 = synth.config("C2", N=8192, Bc=cfg.Bc, causal=cfg.causal)
+            q8, k8, v8 = synth.make_qkv_device(c8, dev)
+            qkv8 = hb.alloc_qkv(c8.B, c8.Hq, c8.Hkv, c8.N, c8.d, dt, dev)
+            out8 = torch.empty((c8.B, c8.Hq, c8.N, c8.d), dtype=torch.float32, device=dev)
+
+            def step8():
+                hb.quantize_qkv(q8, k8, v8, s, inv_s, out=qkv8, d_status=status)
+                hb.attention_fwd(qkv8, c8.causal, Bc=c8.Bc, out_dtype=hb.F32, out=out8, d_status=status)
+
+            for _ in range(3):
+                flush_l2(); step8()
+            torch.cuda.synchronize()
+            ms8 = 0.0
+            for _ in range(20):
+                flush_l2()
+                a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+                a.record(); step8(); b.record()
+                torch.cuda.synchronize()
+                ms8 += a.elapsed_time(b)
+            context["C2_at_N8192_step_tflops"] = attn_flops(c8) * 20 / (ms8 * 1e-3) / 1e12
+            del q8, k8, v8, qkv8, out8
+        assert int(status.item()) == 0
+
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -451,7 +496,7 @@ def main():
                        "parallelism": f"replicated batches x{world}"},
             "frac_of_nominal_peak": {k_: value / world / v_ for k_, v_ in NOMINAL.items()},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-            "quantize": quant, "cpu_baseline": cpu}
+            "quantize": quant, "cpu_baseline": cpu, "context": context}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
