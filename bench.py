@@ -1,7 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the HiFA4 hot path on B200: one step = Smooth-QK + HIF4 quantization of Q/K/V
 followed by the fused 4-bit-operand attention forward (Algorithm 1) over one batch of synthetic
-prefill activations.  Prints ONE JSON line ("Measurement").
+prefill activations.  Prints ONE JSON line: metric, value (whole-job TFLOP/s over the timed steps),
+roofline (attention launch against the measured BF16 tensor peak), quantize split, end-to-end figure
+with host buffers, clocks sampled during the timed region, CPU-oracle baseline and context numbers.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--impl ours|reference]
 
