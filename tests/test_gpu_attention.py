@@ -221,3 +221,24 @@ def test_uneven_head_map_equals_reordered_heads(hb, par):
     mapped128 = hb.attention_fwd(hb.quantize_qkv(q, k, v, q_to_kv=head_map), True, Bc=128)
     mha128 = hb.attention_fwd(hb.quantize_qkv(q, k[:, idx].contiguous(), v[:, idx].contiguous()), True, Bc=128)
     assert torch.equal(mapped128, mha128)
+
+
+@pytest.mark.parametrize("name", ["d128-bc64-causal-gqa", "d256-bc64-mild", "d64-bc64-causal-gqa-ragged"])
+def test_output_dtypes_64_key_kernel(hb, par, name):
+    """FP16 / BF16 outputs of the 64-key kernels are the FP32 output rounded once; reruns are bit-identical;
+    rows past a ragged N are not written."""
+    cfg = SMALL[name]
+    q, k, v = synth.make_qkv(cfg)
+    s, inv_s = par.calibrate(cfg, DEV)
+    qkv = hb.quantize_qkv(q.to(DEV), k.to(DEV), v.to(DEV), s, inv_s)
+    o32 = hb.attention_fwd(qkv, cfg.causal, Bc=64, out_dtype=hb.F32)
+    assert torch.equal(o32, hb.attention_fwd(qkv, cfg.causal, Bc=64, out_dtype=hb.F32))
+    assert torch.isfinite(o32).all()
+    o16 = hb.attention_fwd(qkv, cfg.causal, Bc=64, out_dtype=hb.F16)
+    ob16 = hb.attention_fwd(qkv, cfg.causal, Bc=64, out_dtype=hb.BF16)
+    assert torch.equal(o16, o32.to(torch.float16)) and torch.equal(ob16, o32.to(torch.bfloat16))
+    # a caller-provided output buffer with a guard region after it stays untouched beyond [B,Hq,N,d]
+    n = o32.numel()
+    buf = torch.full((n + 4096,), 7.0, dtype=torch.float32, device=DEV)
+    hb.attention_fwd(qkv, cfg.causal, Bc=64, out_dtype=hb.F32, out=buf[:n].view_as(o32))
+    assert torch.equal(buf[:n].view_as(o32), o32) and bool((buf[n:] == 7.0).all())
