@@ -240,3 +240,21 @@ def test_qmean_is_exact_without_quantization(oracle):
     a = oracle.attention_rows(q, pos, k, v, qmean=0, **kw)
     b = oracle.attention_rows(q, pos, k, v, qmean=1, **kw)
     assert np.max(np.abs(a - b)) < 1e-11
+
+
+def test_p_dtype_flag_is_one_fp16_rounding(oracle):
+    """The FP16-P default and the FP32-P variant differ by exactly one rounding of P: with the same scores
+    and running maxima (the maxima do not depend on P), P16 = float16(P32) element by element (numpy's
+    cast), P32 is an FP32 value, and P32 = fl32(exp2(t)) to FP32 accuracy."""
+    q, k, v, pos = _small(5)
+    kw = dict(causal=True, Bc=64, in_dtype=oracle.F16, dumps=True)
+    _, d16 = oracle.attention_rows(q, pos, k, v, p_dtype=oracle.F16, **kw)
+    _, d32 = oracle.attention_rows(q, pos, k, v, p_dtype=oracle.F32, **kw)
+    assert np.array_equal(d16["m_trace"], d32["m_trace"], equal_nan=True)
+    p16, p32 = d16["p_raw"], d32["p_raw"]
+    assert np.array_equal(p32, p32.astype(np.float32).astype(np.float64))
+    assert np.array_equal(p16, p32.astype(np.float16).astype(np.float64))
+    assert (p16 != p32)[p32 > 0].mean() > 0.9            # the flag does something (masked keys are 0 in both)
+    # and the codes differ in a small fraction of elements only (the two are different functions)
+    frac = (d16["p_codes"] != d32["p_codes"]).mean()
+    assert 0 < frac < 5e-3, frac
