@@ -36,7 +36,8 @@ constexpr int V_OFF = K_OFF + STAGES * K_STAGE;
 constexpr int MISC_OFF = V_OFF + STAGES * V_STAGE;  // barriers, tmem slot, abort flag
 constexpr int XCHG_OFF = MISC_OFF + 256;            // partial row maxima [2 parities][4 splits][128 rows]
 constexpr int XCHG_BYTES = 2 * 4 * 128 * 4;
-constexpr int SMEM_BYTES = XCHG_OFF + XCHG_BYTES + 1024;
+constexpr int STG_OFF = XCHG_OFF + XCHG_BYTES;      // per softmax warp: 8 rows x 128 bytes of output staging
+constexpr int SMEM_BYTES = STG_OFF + 16 * 1024 + 1024;
 constexpr int O_COLS = D + 16, QT_COL = 144, S_COL = 256, TMEM_COLS = 512;
 enum { BAR_QFULL = 0, BAR_QFREE = 2, BAR_KF = 4, BAR_KE = 6, BAR_VF = 8, BAR_VE = 10, BAR_SF = 12,
        BAR_PF = 14, BAR_PV = 16, BAR_X = 17, BAR_QT = 25, N_BARS = 26 };
@@ -479,25 +480,56 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
                 tmem_wait_ld();
                 const float ell = __uint_as_float(lr[0]);
                 const float l16 = f16_round(ell);
+                // O / l as the correctly rounded quotient from the correctly rounded reciprocal and one
+                // correction step (no value here is near the ends of the FP32 range)
+                const float rl = __frcp_rn(l16);
                 if (DBG && dbg_slot >= 0 && row < N && kq == 0) {
                     if (args.dbg.l_out) args.dbg.l_out[dbg_slot * 128 + r_loc] = ell;
                     if (args.dbg.m_out) args.dbg.m_out[dbg_slot * 128 + r_loc] = m_run;
                 }
                 const size_t orow = ((size_t)it.bh_q * N + row) * D + kq * KPT;
+                const uint32_t stage = smem_base + STG_OFF + (uint32_t)warp * 1024u;
 #pragma unroll
                 for (int cc = 0; cc < KPT / 32; ++cc) {
                     uint32_t r[32];
                     tmem_ld32(t_lane + kq * KPT + cc * 32, r);
                     tmem_wait_ld();
-                    if (row < N) {
-                        float o[32];
+                    float o[32];
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] = __fdiv_rn(__uint_as_float(r[i]), l16);
-                        if (args.out_dtype == HIFA4_F32) {
-                            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(args.out) + orow + cc * 32);
+                    for (int i = 0; i < 32; ++i) {
+                        const float a = __uint_as_float(r[i]);
+                        const float q0v = a * rl;
+                        o[i] = fmaf(fmaf(-q0v, l16, a), rl, q0v);
+                    }
+                    if (args.out_dtype == HIFA4_F32) {
+                        // through shared memory, 8 rows at a time, so that a store instruction writes whole
+                        // 128-byte lines
+                        const int c4r = lane & 7, sub = lane >> 3;
+                        float* obase = reinterpret_cast<float*>(args.out) + ((size_t)it.bh_q * N + q0 + quarter * 32) * D +
+                                       kq * KPT + cc * 32 + c4r * 4;
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) dst[i] = make_float4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
-                        } else {
+                        for (int pass = 0; pass < 4; ++pass) {
+                            if ((lane >> 3) == pass) {
+#pragma unroll
+                                for (int c4 = 0; c4 < 8; ++c4)
+                                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};"
+                                                 ::"r"(stage + (lane & 7) * 128 + ((c4 ^ (lane & 7)) << 4)), "f"(o[4 * c4]),
+                                                   "f"(o[4 * c4 + 1]), "f"(o[4 * c4 + 2]), "f"(o[4 * c4 + 3]) : "memory");
+                            }
+                            __syncwarp();
+#pragma unroll
+                            for (int hh = 0; hh < 2; ++hh) {
+                                const int r8 = hh * 4 + sub, rr = pass * 8 + r8;
+                                float4 v;
+                                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                             : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                                             : "r"(stage + r8 * 128 + ((c4r ^ r8) << 4)));
+                                if (q0 + quarter * 32 + rr < N) *reinterpret_cast<float4*>(obase + (size_t)rr * D) = v;
+                            }
+                            __syncwarp();
+                        }
+                    } else if (row < N) {
+                        {
                             uint32_t w[16];
 #pragma unroll
                             for (int i = 0; i < 16; ++i) {
