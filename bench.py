@@ -33,6 +33,7 @@ UNIT = "TFLOP/s"
 NOMINAL = {"fp4": 9000.0, "fp8": 4500.0, "bf16": 2250.0}      # dense TFLOP/s, context only
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture
 # summarised in profiles/attention_fwd_ws_C2.md (bytes per launch; None where not captured)
+NCU_INSTR_PER_WARP_SCORE = {"attention_fwd_ws64_kernel<128>": 17.9}   # profiles/attention_fwd_ws64_C2.md
 NCU_TRAFFIC_BYTES = {("C2-qwen3-8b-4k", 64): 68.70e6, ("C2-qwen3-8b-4k", 128): 67.14e6}
 
 
@@ -468,6 +469,23 @@ def main():
                 "timed_in": "a second pass of the same steps with one event between the two launches "
                             f"({split_step_ms:.4f} ms per step there)",
                 "frac_of_nominal": {k_: achieved / v_ for k_, v_ in NOMINAL.items()}}
+    # The binding resource of the attention kernel is the issue rate of its softmax/quantizer warps, not
+    # the tensor pipe: scores per second against (SMs x 4 schedulers x clock) warp-instructions per second
+    # divided by the warp-instructions the kernel executes per 32 scores (ncu opcode counters, profiles/).
+    n_scores = cfg.B * cfg.Hq * sum(min(cfg.N, ((qb * 128 + 127) // cfg.Bc + 1) * cfg.Bc) if cfg.causal else cfg.N
+                                    for qb in range((cfg.N + 127) // 128)) * 128
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+    sm_hz = (clocks.get("sm_mhz") or 1965.0) * 1e6
+    instr_per_warp_score = NCU_INSTR_PER_WARP_SCORE.get(kern)
+    roofline_alu = None
+    if instr_per_warp_score:
+        peak_scores = sm_count * 4 * sm_hz * 32 / instr_per_warp_score
+        ach_scores = n_scores / (attn_avg_ms * 1e-3)
+        roofline_alu = {"bound": "alu", "kernel": kern, "achieved": ach_scores / 1e9, "peak": peak_scores / 1e9,
+                        "unit": "Gscore/s", "frac": ach_scores / peak_scores,
+                        "instr_per_warp_score": instr_per_warp_score,
+                        "peak_source": f"{sm_count} SMs x 4 schedulers x {sm_hz / 1e6:.0f} MHz (sampled) x 32 lanes / "
+                                       "executed warp instructions per warp-score (ncu)"}
     q_bytes = sum(t.numel() for t in (q, k, v)) * (2 + 0.5625)
     quant = {"avg_ms": sum(quant_ms) / len(quant_ms), "algorithmic_gbs": q_bytes / (sum(quant_ms) / len(quant_ms) * 1e-3) / 1e9,
              "hbm_peak_gbs": peaks["hbm"]}
@@ -498,7 +516,7 @@ def main():
                        "parallelism": f"replicated batches x{world}"},
             "frac_of_nominal_peak": {k_: value / world / v_ for k_, v_ in NOMINAL.items()},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-            "quantize": quant, "cpu_baseline": cpu, "context": context}
+            "roofline_alu": roofline_alu, "quantize": quant, "cpu_baseline": cpu, "context": context}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
