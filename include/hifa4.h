@@ -241,7 +241,11 @@ size_t hifa4_attention_workspace_bytes(const hifa4_shape* shape, const hifa4_att
  *   qkv: buffers filled by hifa4_quantize_qkv for the same shape (only the
  *   *_mma images are read).  out: [B,Hq,N,d] of prm->out_dtype.
  *   workspace: at least hifa4_attention_workspace_bytes() bytes (NULL if 0).
- *   dbg: NULL, or a P-hat dump request. */
+ *   dbg: NULL, or a P-hat dump request.
+ * Scheduling note: for Bc = 64 the grid is launched with programmatic stream
+ * serialization, i.e. its CTAs may become resident while the preceding kernel
+ * of the stream is still draining; they read and write no global memory before
+ * that kernel has completed, so the usual stream order of results holds. */
 int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv,
                         const hifa4_attn_params* prm, void* out, void* workspace,
                         const hifa4_debug* dbg, int* d_status, void* stream);
