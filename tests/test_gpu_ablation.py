@@ -147,12 +147,13 @@ def test_fp32_p_variant_full_size_sampled(hb, par):
     print(par.assert_within_bars(res, "C2 p=f32"))
 
 
-def test_method_components_against_fp32_attention(hb, par):
+@pytest.mark.parametrize("N", [256, 1024, 4096])
+def test_method_components_against_fp32_attention(hb, par, N):
     """End-to-end effect of the components on the outlier inputs, with plain FP32 softmax attention
     (torch, on the unquantized inputs) as the yardstick: Smooth-QK lowers the relative L2 error
     markedly ("Smooth-QK" and the ablation table); the normalizer mode barely moves relative L2 but
     shrinks the output towards the origin by the lost mass (Theorem 1: O_mis = O_con (1 + eps-bar))."""
-    cfg = synth.config("C2", N=1024, Hq=8, Hkv=2, cal_samples=4, cal_tokens=256)
+    cfg = synth.config("C2", N=N, Hq=8, Hkv=2, cal_samples=4, cal_tokens=256)
     q, k, v = (t.to(DEV) for t in synth.make_qkv(cfg))
     s, inv_s = par.calibrate(cfg, DEV)
     kk = k.float().repeat_interleave(cfg.Hq // cfg.Hkv, dim=1)
@@ -170,7 +171,7 @@ def test_method_components_against_fp32_attention(hb, par):
     o_smooth_mis = hb.attention_fwd(smooth, True, Bc=64, normalizer=1)
     e = {n: rel_l2(o) for n, o in (("hifa4", o_hifa4), ("no-smooth", o_nosmooth), ("direct", o_direct),
                                    ("smooth+mismatched", o_smooth_mis))}
-    print(e)
+    print(N, e)
     assert e["hifa4"] < 0.85 * e["no-smooth"] and e["hifa4"] < 0.85 * e["direct"]
     assert abs(e["hifa4"] - e["smooth+mismatched"]) < 0.05 * e["hifa4"]
     # radial contraction of the mismatched output: its projection on the consistent one is below 1
