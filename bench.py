@@ -176,7 +176,9 @@ def run_reference(args, cfg, rank):
     q, k, v = (t.float().numpy() for t in host_inputs(cfg))
     s, inv_s = oracle_scales(cfg)
     t1, cores = oracle_time(cfg, q, k, v, s, inv_s, [0])
-    n_heads = max(1, min(cfg.Hq, int(8.0 / max(t1, 1e-3))))          # about 8 s of CPU work per step
+    # the whole run (warm-up included) gets about two minutes of CPU work, at most 8 s per step
+    per_step = min(8.0, 120.0 / max(args.steps + args.warmup, 1))
+    n_heads = max(1, min(cfg.Hq, int(per_step / max(t1, 1e-3))))
     heads = [int(i * cfg.Hq / n_heads) for i in range(n_heads)]
     for _ in range(args.warmup):
         oracle_time(cfg, q, k, v, s, inv_s, heads[:1])
