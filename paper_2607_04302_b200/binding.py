@@ -299,7 +299,7 @@ def quantize_qkv(q, k, v, s=None, inv_s=None, q_to_kv=None, out: QuantizedQKV | 
     return out
 
 
-def attention_fwd(qkv: QuantizedQKV, causal: bool, Bc: int = 128, out_dtype=F32, out=None,
+def attention_fwd(qkv: QuantizedQKV, causal: bool, Bc: int = 64, out_dtype=F32, out=None,
                   debug_blocks=None, d_status=None, softmax_scale=0.0, Br=128, qmean=False, normalizer=0,
                   p_dtype=F16):
     """Fused attention forward on quantized operands.  Returns out [B,Hq,N,d], or
@@ -330,7 +330,7 @@ def attention_fwd(qkv: QuantizedQKV, causal: bool, Bc: int = 128, out_dtype=F32,
     return (out, dump) if debug_blocks else out
 
 
-def attention_fwd_stats(qkv: QuantizedQKV, causal: bool, n_bins: int, lo: float, hi: float, Bc: int = 128,
+def attention_fwd_stats(qkv: QuantizedQKV, causal: bool, n_bins: int, lo: float, hi: float, Bc: int = 64,
                         out_dtype=F32, hist=None, d_status=None, softmax_scale=0.0, qmean=False, normalizer=0):
     """Attention forward that also adds to the histogram of the per-(row, key tile) mass error of P-hat.
     Returns (out, hist) with hist a device int64 tensor of n_bins + 2 counters (last two: below lo, at or above hi)."""
@@ -354,7 +354,7 @@ def attention_raw_workspace_bytes(B, Hq, Hkv, N, d, in_dtype, causal, Bc, out_dt
     return int(lib().hifa4_attention_raw_workspace_bytes(C.byref(sh), C.byref(prm)))
 
 
-def attention_fwd_raw(q, k, v, s, inv_s, causal: bool, Bc: int = 128, out_dtype=F32, q_to_kv=None,
+def attention_fwd_raw(q, k, v, s, inv_s, causal: bool, Bc: int = 64, out_dtype=F32, q_to_kv=None,
                       out=None, workspace=None, d_status=None, softmax_scale=0.0, qmean=False):
     """Algorithm 1 end to end on raw device tensors (quantize into the workspace, then attend)."""
     B, Hq, N, d = q.shape
