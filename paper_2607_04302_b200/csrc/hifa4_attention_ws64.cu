@@ -17,6 +17,12 @@
 //   d = 128: 256 tensor-memory columns: [O | l] 0..143 (one N = 144 MMA), S 144..207, P-hat
 //            208..239; Q-hat stays in shared memory (SS-form Q K^T).  101 KB of shared memory and
 //            <= 102 registers, so two CTAs share an SM and fill each other's synchronisation gaps.
+// Polls for S(j+1) and PV(j-1) are issued early with test_wait (try_wait blocks while the phase is
+// incomplete); the blocking wait is the fall-back.  Epilogue: O / l by reciprocal plus one correction
+// step, FP32 output through a per-warp 32 x 32 shared-memory transpose (the K stages are idle by then).
+// The grid is launched with programmatic stream serialization: everything before griddepcontrol.wait
+// (barrier set-up, tensor-memory allocation) may overlap the tail of the preceding kernel.
+// Template flags: P-hat dump, FP32-P variant, Q-Mean (key sums staged in shared memory by the producer).
 // Every wait is bounded (see hifa4_attention_ws.cu for the failure protocol).
 #include "hifa4_attention.cuh"
 
