@@ -290,6 +290,14 @@ def main():
 
     sampler = ClockSampler(local_rank)
     sampler.start()
+    # spin-up (untimed, before the W warm-up steps): a fresh process on a fresh box starts with idle
+    # clocks and unloaded modules; a quarter of a second of the same steps brings both up
+    t_spin = time.perf_counter() + 0.25
+    while time.perf_counter() < t_spin:
+        for _ in range(10):
+            flush_l2()
+            step()
+        torch.cuda.synchronize()
     for _ in range(args.warmup):
         flush_l2()
         step()
