@@ -134,10 +134,9 @@ def smooth_quantize(x: np.ndarray, scale, dtype: int, axis_tokens: bool = False)
     return hif4_quantize_rows(y)
 
 
-def qmean_quantize(x: np.ndarray, scale, dtype: int):
-    """Algorithm 1 lines 1-3 for Q with the Q-Mean auxiliary: smooth, subtract the per-token mean
-    (kept in FP16), round to the activation dtype, HIF4 along channels.
-    x [..., N, d]; returns (codes, meta, deq, mu [..., N])."""
+def qmean_rows(x: np.ndarray, scale, dtype: int):
+    """Algorithm 1 lines 1-2 for Q: smooth, subtract the per-token mean (kept in FP16), round to the
+    activation dtype.  x [..., N, d]; returns (q_z float64 [..., N, d], mu [..., N])."""
     x = np.ascontiguousarray(x, np.float32)
     d = x.shape[-1]
     rows = x.size // d
@@ -146,6 +145,13 @@ def qmean_quantize(x: np.ndarray, scale, dtype: int):
     sc = None if scale is None else np.ascontiguousarray(scale, np.float32)
     lib().hifa4_oracle_qmean_rows(_p(x, C.c_float), C.c_long(rows), C.c_int(d), _p(sc, C.c_float),
                                   C.c_int(dtype), _p(y, C.c_double), _p(mu, C.c_double))
+    return y, mu
+
+
+def qmean_quantize(x: np.ndarray, scale, dtype: int):
+    """Algorithm 1 lines 1-3 for Q with the Q-Mean auxiliary: qmean_rows, then HIF4 along channels.
+    x [..., N, d]; returns (codes, meta, deq, mu [..., N])."""
+    y, mu = qmean_rows(x, scale, dtype)
     return hif4_quantize_rows(y) + (mu,)
 
 

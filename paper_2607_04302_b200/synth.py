@@ -109,7 +109,8 @@ def make_calibration(cfg: Config, samples: int | None = None, tokens: int | None
 def make_qkv_device(cfg: Config, device, seed: int | None = None):
     """Same distribution drawn on the device (for sizes too large to draw on the host).
 
-    The values differ from make_qkv (a different generator); use it for timing only."""
+    The values differ from make_qkv (a different generator).  Used for timing and for parity on sampled
+    rows at sizes where only those rows and their K/V head are copied back to the host."""
     gen = torch.Generator(device=device).manual_seed(cfg.seed if seed is None else seed)
     dt = torch_dtype(cfg)
 

@@ -2,6 +2,7 @@
 Theorem 1's closed forms, and the invariants the method states."""
 import numpy as np
 import pytest
+import torch
 
 from paper_2607_04302_b200 import synth
 
@@ -240,6 +241,62 @@ def test_qmean_is_exact_without_quantization(oracle):
     a = oracle.attention_rows(q, pos, k, v, qmean=0, **kw)
     b = oracle.attention_rows(q, pos, k, v, qmean=1, **kw)
     assert np.max(np.abs(a - b)) < 1e-11
+
+
+def _cast16(x32: np.ndarray, dtype: str) -> np.ndarray:
+    """float32 array -> 16-bit format and back, by the library casts (numpy float16, torch bfloat16)."""
+    if dtype == "fp16":
+        return x32.astype(np.float16).astype(np.float64)
+    return torch.from_numpy(np.ascontiguousarray(x32)).to(torch.bfloat16).to(torch.float64).numpy()
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_smooth_apply_rounds_the_fp32_product_once_to_the_activation_dtype(oracle, dtype):
+    """Algorithm 1 line 1 with a 16-bit activation: the smoothed value is the FP32 product of the stored
+    activation and the factor, rounded once to the activation dtype (Appendix: the smoothed tensor is a
+    transient 16-bit activation).  Pinned against numpy's float32 multiply and the library casts, on
+    inputs where the rounding matters: skipping it, or rounding to the other 16-bit format, fails."""
+    rng = np.random.default_rng(11)
+    x = _cast16(rng.standard_normal((96, 128)).astype(np.float32) * 3.0, dtype).astype(np.float32)
+    s = np.exp(rng.standard_normal(128) * 0.7).astype(np.float32)
+    want = _cast16(x * s, dtype)                                   # numpy multiplies float32 in float32
+    got = oracle.smooth_apply(x, s, oracle.F16 if dtype == "fp16" else oracle.BF16)
+    assert np.array_equal(got, want)
+    exact = x.astype(np.float64) * s.astype(np.float64)
+    assert (want != exact).mean() > 0.9                            # the rounding is not a no-op here
+    other = _cast16(x * s, "bf16" if dtype == "fp16" else "fp16")
+    assert (want != other).mean() > 0.5                            # and the two formats differ on this data
+    # no factor: the activation passes through untouched
+    assert np.array_equal(oracle.smooth_apply(x, None, oracle.F16), x.astype(np.float64))
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_qmean_vectors_in_fp16_and_mean_free_query_in_the_activation_dtype(oracle, dtype):
+    """Algorithm 1 lines 2 and 6 in the deployed precision (Appendix, "Q-Mean GEMV and coordinate
+    consistency"): mu_i = FP16(mean_c q~_ic) and ksum_j = FP16(sum_c k~_jc) from exact sums of the smoothed
+    16-bit activations, Q_z = q~ - mu rounded once to the activation dtype.  Pinned against numpy double
+    sums and the library casts."""
+    rng = np.random.default_rng(12)
+    odt = oracle.F16 if dtype == "fp16" else oracle.BF16
+    x = _cast16(rng.standard_normal((80, 128)).astype(np.float32) + 0.6, dtype).astype(np.float32)
+    s = np.exp(rng.standard_normal(128) * 0.5).astype(np.float32)
+    xt = _cast16(x * s, dtype)                                     # smoothed activation (line 1), float64 holder
+    mu_want = xt.sum(1) / 128
+    mu_want = mu_want.astype(np.float16).astype(np.float64)
+    qz_want = _cast16((xt - mu_want[:, None]).astype(np.float32), dtype)
+    # the difference of a 16-bit value and an FP16 value fits float32 exactly here (|values| < 2^5, bits > 2^-24)
+    assert np.array_equal((xt - mu_want[:, None]).astype(np.float32).astype(np.float64), xt - mu_want[:, None])
+    qz, mu = oracle.qmean_rows(x, s, odt)
+    assert np.array_equal(mu, mu_want) and np.array_equal(qz, qz_want)
+    assert np.abs(mu_want).min() > 0.05                            # the mean matters on this data
+    assert (qz_want != xt - mu_want[:, None]).mean() > 0.2         # so does the rounding of Q_z
+    ks_want = xt.sum(1).astype(np.float16).astype(np.float64)
+    assert np.array_equal(oracle.ksum_rows(x, s, odt), ks_want)
+    assert (ks_want != xt.sum(1)).mean() > 0.5                     # FP16 rounding of the key sums is visible
+    # qmean_quantize = the same Q_z through the HIF4 encoder
+    c, m, dq, mu2 = oracle.qmean_quantize(x, s, odt)
+    c2, m2, dq2 = oracle.hif4_quantize_rows(qz_want)
+    assert np.array_equal(c, c2) and np.array_equal(m, m2) and np.array_equal(dq, dq2) and np.array_equal(mu2, mu_want)
 
 
 def test_p_dtype_flag_is_one_fp16_rounding(oracle):
