@@ -37,11 +37,13 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
     const int N = args.N;
     const int row = q0 + tid;                             // this thread's query row
 
-    // a CTA that starts after another one reported a failure does nothing
-    if (args.d_status && *reinterpret_cast<volatile int*>(args.d_status) != 0) return;
-
     // ---- set-up: barriers, tensor memory, ones rows under every V^T chunk
+    volatile int* dead_flag = reinterpret_cast<volatile int*>(smem_gen + C::BAR_OFF + 40);
     if (tid == 0) {
+        // A CTA that starts after another one reported a failure does nothing.  One thread reads the status
+        // word and publishes the verdict through shared memory: every thread then takes the same path, and
+        // that path still frees the tensor memory allocated below.
+        *dead_flag = (args.d_status && *reinterpret_cast<volatile int*>(args.d_status) != 0) ? 1 : 0;
         tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_k); tma_prefetch_desc(&tmap_v);
         mbar_init(bar_q, 1); mbar_init(bar_kv, 1); mbar_init(bar_mma, 1);
         fence_barrier_init();
@@ -68,6 +70,7 @@ attention_fwd_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_co
     bool ok = true;
     uint32_t mma_phase = 0;
     int fail_site = 0;
+    if (*dead_flag) goto done;
 
     if (tid == 0) {
         mbar_expect_tx(bar_q, C::KSUB * C::Q_SUB_BYTES);
@@ -297,14 +300,15 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 static EncodeTiledFn get_encode()
 {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
+    // initialised once, thread-safe (a function-local static); null if the driver lacks the entry point
+    static const EncodeTiledFn fn = [] {
         void* p = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
             qres == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-    }
+            return (EncodeTiledFn)p;
+        return (EncodeTiledFn) nullptr;
+    }();
     return fn;
 }
 
@@ -330,12 +334,8 @@ static int launch_cfg(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArg
     if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, D, BC)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, D, sh.N, D)) return HIFA4_ERR_CUDA;
     auto kern = attention_fwd_kernel<D, BC, AUX>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
-            return HIFA4_ERR_CUDA;
-        attr_set = true;
-    }
+    static SmemOptIn opt_in;
+    if (!opt_in.ensure(kern, C::SMEM_BYTES)) return HIFA4_ERR_CUDA;
     dim3 grid((sh.N + 127) / 128, sh.Hq, sh.B);
     kern<<<grid, 128, C::SMEM_BYTES, st>>>(mq, mk, mv, args);
     count_launch();

@@ -113,8 +113,6 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     constexpr int W_TMA = NSW, W_MMA = NSW + 1;
     constexpr int KPT = BC / KS;                // keys per thread and tile
     constexpr int NU = KPT / 8;                 // level-2 units per thread
-    if (args.d_status && *reinterpret_cast<volatile int*>(args.d_status) != 0) return;
-
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -134,7 +132,10 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     const int n_my = sched.count();             // items of this CTA
 
     if (tid == 0) {
-        *abort_flag = 0;
+        // A CTA that starts after another one reported a failure does nothing.  One thread reads the status
+        // word and publishes the verdict through shared memory, so that all roles of the CTA agree on it
+        // and leave through the common exit that frees tensor memory.
+        *abort_flag = (args.d_status && *reinterpret_cast<volatile int*>(args.d_status) != 0) ? 2 : 0;
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar(BAR_QFULL + s), 1); mbar_init(bar(BAR_QFREE + s), NSW);
             mbar_init(bar(BAR_KF + s), 1); mbar_init(bar(BAR_KE + s), 1);
@@ -157,6 +158,7 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    const bool dead = *abort_flag != 0;
 
     auto fail = [&](int site) {
         *abort_flag = 1;
@@ -165,7 +167,9 @@ attention_fwd_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid
 
     // Tiles are numbered globally across the items of this CTA (g = 0, 1, ...): ring stages, S buffers
     // and barrier phases follow g, so the tile stream runs through item boundaries without a drain.
-    if (warp == W_TMA) {
+    if (dead) {
+        // fall through to the common exit
+    } else if (warp == W_TMA) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             int g = 0;
@@ -565,19 +569,12 @@ static int launch_ws(const hifa4_shape& sh, const CUtensorMap& mq, const CUtenso
                      const AttnArgs& args, cudaStream_t st)
 {
     auto kern = attention_fwd_ws_kernel<KS, DBG, QM>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ws::SMEM_BYTES) != cudaSuccess)
-            return HIFA4_ERR_CUDA;
-        attr_set = true;
-    }
-    static int sm_count = 0;
-    if (!sm_count) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
-            return HIFA4_ERR_CUDA;
-    }
+    static SmemOptIn opt_in;
+    if (!opt_in.ensure(kern, ws::SMEM_BYTES)) return HIFA4_ERR_CUDA;
+    int dev = 0, sm_count = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0)
+        return HIFA4_ERR_CUDA;
     const long long n_items = (long long)((sh.N + 127) / 128) * sh.Hq * sh.B;
     dim3 grid((unsigned)(n_items < sm_count ? n_items : sm_count));     // persistent: one CTA per SM
     kern<<<grid, (4 * KS + 2) * 32, ws::SMEM_BYTES, st>>>(mq, mk, mv, args);

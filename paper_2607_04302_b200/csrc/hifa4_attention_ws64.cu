@@ -141,6 +141,9 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     // become resident and set themselves up as SMs drain); nothing the predecessor wrote is touched
     // before this point.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // The status word was read before the wait; a non-zero value may be one that the preceding work in the
+    // stream has cleared since, so only that (rare) verdict is confirmed by a second read.
+    if (tid == 0 && *abort_flag) *abort_flag = *reinterpret_cast<volatile int*>(args.d_status) != 0 ? 2 : 0;
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
@@ -563,12 +566,8 @@ static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnAr
     if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, DH, C::BC)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, DH, sh.N, DH)) return HIFA4_ERR_CUDA;
     auto kern = attention_fwd_ws64_kernel<DH, DBG, PF32, QM>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES) != cudaSuccess)
-            return HIFA4_ERR_CUDA;
-        attr_set = true;
-    }
+    static SmemOptIn opt_in;
+    if (!opt_in.ensure(kern, C::SMEM_BYTES)) return HIFA4_ERR_CUDA;
     dim3 grid((unsigned)(((sh.N + 127) / 128) * sh.Hq * sh.B));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;

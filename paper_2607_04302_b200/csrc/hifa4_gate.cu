@@ -109,13 +109,8 @@ cudaError_t launch_gate(int dtype, const void* k_cal, long long nk, const float*
     double* gate = reinterpret_cast<double*>(reinterpret_cast<char*>(gate_ws) + HIST_BINS * sizeof(uint32_t));
     cudaError_t e = cudaMemsetAsync(hist, 0, HIST_BINS * sizeof(uint32_t), st);
     if (e != cudaSuccess) return e;
-    static bool attr_set = false;
-    if (!attr_set) {
-        e = cudaFuncSetAttribute(abs_hist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)(HIST_BINS * sizeof(uint32_t)));
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
+    static SmemOptIn opt_in;
+    if (!opt_in.ensure(abs_hist_kernel, (int)(HIST_BINS * sizeof(uint32_t)))) return cudaErrorInvalidValue;
     const long long n_vec = nk / 8;
     int sms = 148;
     int dev = 0;

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <mutex>
 #include "../../include/hifa4.h"
 
 namespace hifa4 {
@@ -9,6 +10,26 @@ namespace hifa4 {
 struct HeadMap;
 
 void count_launch();
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) holds for one device only: each launcher keeps one of
+// these per kernel instantiation and opts in once per device, under a lock (host threads may race).
+struct SmemOptIn {
+    static constexpr int MAX_DEVICES = 64;
+    std::mutex m;
+    bool done[MAX_DEVICES] = {};
+    template <class Kernel>
+    bool ensure(Kernel kern, int bytes)
+    {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return false;
+        std::lock_guard<std::mutex> lock(m);
+        if (!done[dev]) {
+            if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+            done[dev] = true;
+        }
+        return true;
+    }
+};
 
 // One launch for Q, K and V (null inputs are skipped).  out.q_mu / out.k_sum non-null: Q-Mean
 // (subtract the per-row mean of Q and write it; write the per-row channel sum of K).

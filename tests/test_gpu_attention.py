@@ -256,3 +256,25 @@ def test_output_dtypes_64_key_kernel(hb, par, name):
     buf = torch.full((n + 4096,), 7.0, dtype=torch.float32, device=DEV)
     hb.attention_fwd(qkv, cfg.causal, Bc=64, out_dtype=hb.F32, out=buf[:n].view_as(o32))
     assert torch.equal(buf[:n].view_as(o32), o32) and bool((buf[n:] == 7.0).all())
+
+
+@pytest.mark.parametrize("d,Bc,normalizer", [(128, 64, 0), (256, 64, 0), (128, 128, 0), (64, 128, 0), (128, 64, 1)])
+def test_nonzero_status_word_makes_every_kernel_family_a_no_op(hb, par, d, Bc, normalizer):
+    """A call whose status word already holds an error does nothing: every CTA reads the word once,
+    all of its roles agree on the verdict and leave through the common exit (which still frees tensor
+    memory), the output buffer is untouched and the word is preserved.  The next ordinary call on the
+    same device works, i.e. no tensor memory leaked and no barrier was left armed."""
+    cfg = synth.config("C3", N=384, Hq=2, Hkv=1, d=d, Bc=Bc)
+    q, k, v = (t.to(DEV) for t in synth.make_qkv(cfg))
+    qkv = hb.quantize_qkv(q, k, v)
+    status = torch.full((1,), 77, dtype=torch.int32, device=DEV)
+    out = torch.full((cfg.B, cfg.Hq, cfg.N, cfg.d), 5.0, dtype=torch.float32, device=DEV)
+    for _ in range(3):                                         # several launches: leaked tensor memory would block
+        hb.attention_fwd(qkv, True, Bc=Bc, out=out, d_status=status, normalizer=normalizer)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 77 and bool((out == 5.0).all())
+    status.zero_()
+    good = hb.attention_fwd(qkv, True, Bc=Bc, d_status=status, normalizer=normalizer)
+    hb.attention_fwd(qkv, True, Bc=Bc, out=out, d_status=status, normalizer=normalizer)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(out, good) and torch.isfinite(out).all()
