@@ -162,8 +162,8 @@ __device__ __forceinline__ float p_of_score(float acc, float c1, float mL)
 //   v = fma(y, S/4, -magic*S/4)  = m * 2^k * S/4, the dequantized value, no rounding
 // The shift k of a 4-key subgroup with maximum At is read off float bit patterns:
 //   need = max(bits(At) - bits(1.75 S) - 1 + 2^23, 0) >> 23   (0, 1 or 2)
-// and the pair rule "level-2 bit = 1 iff max(need) = 2 or min(need) >= 1" is a = (n0 + n1 + 2) >> 2,
-// k = max(need, a).  Multiplications, additions and FMAs run two elements at a time (f32x2).
+// (the shifts of the two subgroups of a level-2 unit are then combined by exp_quantize_units).
+// Multiplications, additions and FMAs run two elements at a time (f32x2).
 struct PQuantConst {              // per (row, 64-key group, tile) constants of the fused quantizer
     uint64_t c1c1, nml, inv44, s44;
     uint32_t c0_bits, s4_bits;
@@ -205,11 +205,17 @@ __device__ __forceinline__ void exp_unit(const float (&acc)[NU * 8], int u, cons
 // Units U0..U1-1 of a thread's NU units: acc -> P (FP16) -> P-hat image words w[4u..4u+3].
 // The exponentials of unit u+1 are issued before unit u is quantized, so that the MUFU latency of
 // one unit hides behind the ALU/FMA work of the previous one.
+// A unit is two 4-key subgroups t = 0, 1 with shifts k_t = max(need_t, need_other - 1) (that is the
+// pair rule: the level-2 bit is set iff max(need) = 2 or min(need) >= 1, and a subgroup that needs no
+// shift of its own still gets one when its partner needs two).  On bit patterns, with
+// x_t = max(bits(At_t) + tadd, 0) = need_t * 2^23 + fraction: k_t * 2^23 = max(x_t, x_other - 2^23)
+// with the fraction masked off.  The packed operations pair key i of subgroup 0 with key i of
+// subgroup 1, so that one pair of per-subgroup constants (magic, c) serves four packed operations.
 template <int NU, int U0, int U1, bool DBG, bool PF32 = false>
 __device__ __forceinline__ void exp_quantize_units(const float (&acc)[NU * 8], const PQuantConst& k, bool zero_group,
                                                    uint32_t (&w)[NU * 4], uint8_t* dump_codes, float* dump_step)
 {
-    const uint32_t MAGIC_BITS = 0x4B400000u;                               // 1.5 * 2^23
+    const int MAGIC_BITS = 0x4B400000;                                    // 1.5 * 2^23
     float pn[8];
     exp_unit<NU, PF32>(acc, U0, k, pn);
 #pragma unroll
@@ -220,31 +226,36 @@ __device__ __forceinline__ void exp_quantize_units(const float (&acc)[NU * 8], c
         if (u + 1 < U1) exp_unit<NU, PF32>(acc, u + 1, k, pn);
         const float At0 = fmaxf(max3(p[0], p[1], p[2]), p[3]);
         const float At1 = fmaxf(max3(p[4], p[5], p[6]), p[7]);
-        const int n0 = max((int)__float_as_uint(At0) + k.tadd, 0) >> 23;
-        const int n1 = max((int)__float_as_uint(At1) + k.tadd, 0) >> 23;
-        const int a = (n0 + n1 + 2) >> 2;
+        const int x0 = max((int)__float_as_uint(At0) + k.tadd, 0);
+        const int x1 = max((int)__float_as_uint(At1) + k.tadd, 0);
+        const int ks0 = max(x0, x1 - (1 << 23)) & (int)0xFF800000;
+        const int ks1 = max(x1, x0 - (1 << 23)) & (int)0xFF800000;
+        const uint64_t mm = pack2(__int_as_float(MAGIC_BITS + ks0), __int_as_float(MAGIC_BITS + ks1));
+        const uint64_t cc = pack2(__int_as_float((int)k.c0_bits + ks0), __int_as_float((int)k.c0_bits + ks1));
+        float v[8];
+        uint64_t y[4];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const uint32_t ks = (uint32_t)max(h ? n1 : n0, a) << 23;
-            const float magic = __uint_as_float(MAGIC_BITS + ks);
-            const float ck = __uint_as_float(k.c0_bits + ks);
-            const uint64_t mm = pack2(magic, magic), cc = pack2(ck, ck);
-            float v0, v1, v2, v3;
-            const uint64_t y01 = add2(mul2_rz(pack2(p[4 * h], p[4 * h + 1]), k.inv44), mm);
-            const uint64_t y23 = add2(mul2_rz(pack2(p[4 * h + 2], p[4 * h + 3]), k.inv44), mm);
-            unpack2(fma2(y01, k.s44, cc), v0, v1);
-            unpack2(fma2(y23, k.s44, cc), v2, v3);
-            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h]) : "f"(v1), "f"(v0));
-            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + 2 * h + 1]) : "f"(v3), "f"(v2));
-            if (DBG) {
-                float y0, y1, y2, y3;
-                unpack2(y01, y0, y1);
-                unpack2(y23, y2, y3);
-                if (dump_step) dump_step[2 * u + h] = zero_group ? 0.f : __uint_as_float(k.s4_bits + ks);
-                if (dump_codes)
+        for (int i = 0; i < 4; ++i) {
+            y[i] = add2(mul2_rz(pack2(p[i], p[4 + i]), k.inv44), mm);
+            unpack2(fma2(y[i], k.s44, cc), v[i], v[4 + i]);
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + i]) : "f"(v[2 * i + 1]), "f"(v[2 * i]));
+        if (DBG) {
+            float c[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) unpack2(y[i], c[i], c[4 + i]);
+            if (dump_step) {
+                dump_step[2 * u] = zero_group ? 0.f : __int_as_float((int)k.s4_bits + ks0);
+                dump_step[2 * u + 1] = zero_group ? 0.f : __int_as_float((int)k.s4_bits + ks1);
+            }
+            if (dump_codes) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
                     reinterpret_cast<uint32_t*>(dump_codes)[2 * u + h] =
-                        (__float_as_uint(y0) & 15u) | ((__float_as_uint(y1) & 15u) << 8) |
-                        ((__float_as_uint(y2) & 15u) << 16) | ((__float_as_uint(y3) & 15u) << 24);
+                        (__float_as_uint(c[4 * h]) & 15u) | ((__float_as_uint(c[4 * h + 1]) & 15u) << 8) |
+                        ((__float_as_uint(c[4 * h + 2]) & 15u) << 16) | ((__float_as_uint(c[4 * h + 3]) & 15u) << 24);
             }
         }
     }
@@ -280,7 +291,7 @@ bool make_bf16_map(CUtensorMap* m, void* base, uint64_t heads, uint64_t rows, ui
 // Warp-specialised kernel for d = 128, Bc = 128 (hifa4_attention_ws.cu).
 int launch_attention_ws(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st);
 
-// Warp-specialised kernels for Bc = 64, d = 128 or 256 (hifa4_attention_ws64.cu).
+// Warp-specialised kernels for Bc = 64, d = 64, 128 or 256 (hifa4_attention_ws64.cu).
 int launch_attention_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st);
 
 }  // namespace hifa4

@@ -1,22 +1,34 @@
 // Warp-specialised HiFA4 attention forward for Bc = 64 (Algorithm 1 lines 4-13), d = 64, 128 or 256.
 //
 // One CTA = 128 query rows of one (batch, query head), 10 warps:
-//   warps 0-7  softmax / quantize: warp w owns rows 32*(w%4).. of the tile and keys 32*(w/4).. of
-//              every 64-key tile, i.e. half of the tile's single HIF4 group per thread; for the row
-//              maximum each thread also reads the other half of its row from tensor memory (cheaper
-//              than an exchange between the two threads: a poll of an mbarrier costs > 100 clk)
-//   warp 8     TMA producer: Q once, then K and V^T tiles through two-stage rings
-//   warp 9     tcgen05 issuer
+//   warps 0-7  softmax / quantize, one thread per query row and key tile: warps 0-3 own the even key
+//              tiles, warps 4-7 the odd ones (warp w: rows 32*(w%4).., its tensor-memory lane quarter).
+//              The two groups run half a period apart, so that on every scheduler one warp is in its
+//              issue-bound phase (exponentials, quantizer) while the other one sits in a latency-bound
+//              phase (tensor-memory loads and stores, barrier hand-offs); the running maximum of a row
+//              passes from the owner of tile j to the owner of tile j+1 through shared memory, early in
+//              tile j (it is known as soon as the row maximum of S(j) is)
+//   warp 8     one thread: TMA loads of Q and of the K tiles (two-stage ring), tcgen05 issuer of S = Q K^T
+//   warp 9     one thread: TMA loads of the V^T tiles (two-stage ring), issuer of [O | l] += P-hat [V | 1]
+// Each of the two issues its MMA, waits for it to complete (which frees the tile's stage) and refills the
+// stage two tiles ahead; the next MMA of the same kind cannot start earlier anyway (the next S needs the
+// softmax warps to have pulled this S, the next P V needs the P-hat that follows this P V).
+// Each MMA waits on ONE barrier: the barrier that releases S of a tile collects the bytes of the K tile
+// (TMA transaction count) and the eight "S is in registers" arrivals of the softmax warps, the one that
+// releases P V collects the bytes of the V^T tile and the eight "P-hat stored, history rescaled"
+// arrivals.  The two issuers run independently: a late P V never delays the next S (device timestamps
+// of a single in-order issuer showed S(j+1) issued 1500 clk after it could have been).
 // S has a single buffer that is released early: the softmax warps pull S(j) into registers and
-// signal it free, and S(j+1) = Q K^T runs on the tensor pipe while they work on tile j; the BF16
-// image of P-hat has its own tensor-memory columns and is the A operand of the PV MMA.
+// signal it free, and S(j+1) runs on the tensor pipe while they work on tile j; the BF16 image of P-hat
+// has its own tensor-memory columns and is the A operand of the P V MMA.
+// One tile is one 64-key HIF4 group of P per row, held by one thread: no row statistic is computed twice.
 //   d = 256: 512 tensor-memory columns: [O | l] 0..271 (an N = 256 MMA for the channels, an N = 16
 //            MMA on the same A operand for the ones block), Q-hat image 272..399 (A operand of
 //            Q K^T from tensor memory), S 400..463, P-hat 464..495.  One CTA per SM.
 //   d = 64:  as d = 128 with [O | l] 0..79 (one N = 80 MMA); 53 KB of shared memory.
 //   d = 128: 256 tensor-memory columns: [O | l] 0..143 (one N = 144 MMA), S 144..207, P-hat
-//            208..239; Q-hat stays in shared memory (SS-form Q K^T).  101 KB of shared memory and
-//            <= 102 registers, so two CTAs share an SM and fill each other's synchronisation gaps.
+//            208..239; Q-hat stays in shared memory (SS-form Q K^T).  101 KB of shared memory, so two
+//            CTAs share an SM and fill each other's synchronisation gaps.
 // Polls for S(j+1) and PV(j-1) are issued early with test_wait (try_wait blocks while the phase is
 // incomplete); the blocking wait is the fall-back.  Epilogue: O / l by reciprocal plus one correction
 // step, FP32 output through a per-warp 32 x 32 shared-memory transpose (the K stages are idle by then).
@@ -28,17 +40,11 @@
 
 namespace hifa4 {
 
-#ifndef HIFA4_WS64_KS128
-#define HIFA4_WS64_KS128 2
-#endif
-#ifndef HIFA4_WS64_KS256
-#define HIFA4_WS64_KS256 2
-#endif
 template <int D_>
 struct WS64 {
-    static constexpr int D = D_, BC = 64, STAGES = 2, KS = (D_ == 128) ? HIFA4_WS64_KS128 : (D_ == 256 ? HIFA4_WS64_KS256 : 2);
-    static constexpr int NSW = 4 * KS, THREADS = (NSW + 2) * 32, W_TMA = NSW, W_MMA = NSW + 1;
-    static constexpr int KPT = BC / KS, NU = KPT / 8;       // 32 keys = 4 level-2 units per thread and tile
+    static constexpr int D = D_, BC = 64, STAGES = 2;
+    static constexpr int NSW = 8, THREADS = (NSW + 2) * 32, W_QK = NSW, W_PV = NSW + 1;   // two groups of 4 softmax warps
+    static constexpr int NU = BC / 8;                       // 8 level-2 units (64 keys) per thread and tile
     static constexpr int QSUB = D / 64;                     // 64-channel sub-tiles of Q and K
     static constexpr int Q_BYTES = QSUB * 16384;
     static constexpr int K_SUB = BC * 128;                  // 64 keys x 64 channels
@@ -49,7 +55,8 @@ struct WS64 {
     static constexpr int V_OFF = K_OFF + STAGES * K_STAGE;
     static constexpr int MISC_OFF = V_OFF + STAGES * V_STAGE;
     static constexpr int KSUM_OFF = MISC_OFF + 256;         // Q-Mean: channel sums of the tile's 64 keys, two stages
-    static constexpr int SMEM_BYTES = KSUM_OFF + STAGES * 256 + 1024;
+    static constexpr int MX_OFF = KSUM_OFF + STAGES * 256;  // running maxima handed from tile j to tile j+1: [2][128] floats
+    static constexpr int SMEM_BYTES = MX_OFF + 2 * 512 + 1024;
     static constexpr int O_COLS = D + 16;
     static constexpr bool Q_IN_TMEM = (D == 256);
     static constexpr int QT_COL = 272;                      // d = 256 only
@@ -59,20 +66,46 @@ struct WS64 {
     static constexpr int CTAS_PER_SM = (D == 256) ? 1 : 2;
 };
 namespace ws64 {
-enum { BAR_Q = 0, BAR_KF = 1, BAR_KE = 3, BAR_VF = 5, BAR_VE = 7, BAR_SF = 9, BAR_SFREE = 10, BAR_PF = 11,
-       BAR_PV = 12, BAR_KSF = 13, BAR_QT = 17, N_BARS = 18 };
+// Index s = tile % 2 everywhere.  QKGO[s]: K stage s has landed and S is free (4 arrivals + 1 + bytes); PVGO[s]:
+// V^T stage s has landed, the image of P-hat is stored and [O | l] rescaled (4 arrivals + 1 + bytes); KE / VE:
+// stage free (MMA commit); SF[s]: S complete; PV[s]: P V complete; MR[s]: running maxima after the tile
+// published (4 arrivals); KSF[s]: Q-Mean key sums landed; QT: Q-hat image copied to tensor memory.
+// Two barriers per kind because each group of softmax warps sees every second tile only: a parity wait
+// must observe every phase of its barrier.
+enum { BAR_Q = 0, BAR_QKGO = 1, BAR_KE = 3, BAR_PVGO = 5, BAR_VE = 7, BAR_SF = 9, BAR_PV = 11, BAR_KSF = 13,
+       BAR_MR = 15, BAR_QT = 17, N_BARS = 18 };
 constexpr uint32_t WAIT_POLLS = 1u << 20;
 }  // namespace ws64
 
+// Bounded wait with non-blocking polls (softmax warps and issuers: a late wake-up sits on the critical path,
+// and a thread suspended in try_wait was seen to notice a completed phase about 1000 clk late).
 static __device__ __forceinline__ bool wait64(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
-    for (uint32_t i = 0; i < ws64::WAIT_POLLS / 64; ++i) {
 #pragma unroll 1
-        for (int j = 0; j < 64; ++j)
-            if (mbar_try_wait(bar, parity)) return true;
+    for (uint32_t i = 0; i < ws64::WAIT_POLLS; ++i) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if ((i & 63u) == 63u && *abort_flag) return false;
+    }
+    return false;
+}
+// Bounded wait of the producer warp, which waits most of the time and has slack: the hardware may keep the
+// thread suspended for a few microseconds per poll (it wakes when the phase completes).
+static __device__ __forceinline__ bool wait_idle(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+#pragma unroll 1
+    for (uint32_t i = 0; i < ws64::WAIT_POLLS / 4; ++i) {
+        if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
         if (*abort_flag) return false;
     }
     return false;
+}
+// One arrival from lane 0 of a converged warp, without a branch.
+static __device__ __forceinline__ void arrive_lane0(uint32_t bar, int lane)
+{
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "setp.eq.s32 p, %1, 0;\n\t"
+                 "@p mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}"
+                 ::"r"(bar), "r"(lane) : "memory");
 }
 
 template <int DH, bool DBG, bool PF32, bool QM>
@@ -82,8 +115,8 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
 {
     using namespace ws64;
     using C = WS64<DH>;
-    constexpr int D = C::D, BC = C::BC, STAGES = C::STAGES, KS = C::KS, NSW = C::NSW, THREADS = C::THREADS;
-    constexpr int W_TMA = C::W_TMA, W_MMA = C::W_MMA, KPT = C::KPT, NU = C::NU, QSUB = C::QSUB;
+    constexpr int D = C::D, BC = C::BC, STAGES = C::STAGES, NSW = C::NSW, THREADS = C::THREADS;
+    constexpr int W_QK = C::W_QK, W_PV = C::W_PV, NU = C::NU, QSUB = C::QSUB;
     constexpr int Q_BYTES = C::Q_BYTES, K_SUB = C::K_SUB, K_STAGE = C::K_STAGE, V_STAGE = C::V_STAGE;
     constexpr int O_COLS = C::O_COLS, QT_COL = C::QT_COL, S_COL = C::S_COL, P_COL = C::P_COL, TMEM_COLS = C::TMEM_COLS;
 
@@ -119,17 +152,17 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         const int status_now = args.d_status ? *reinterpret_cast<volatile int*>(args.d_status) : 0;
         mbar_init(bar(BAR_Q), 1);
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(bar(BAR_KF + s), 1); mbar_init(bar(BAR_KE + s), 1);
-            mbar_init(bar(BAR_VF + s), 1); mbar_init(bar(BAR_VE + s), 1);
+            mbar_init(bar(BAR_QKGO + s), 5); mbar_init(bar(BAR_KE + s), 1);
+            mbar_init(bar(BAR_PVGO + s), 5); mbar_init(bar(BAR_VE + s), 1);
+            mbar_init(bar(BAR_SF + s), 1); mbar_init(bar(BAR_PV + s), 1);
+            mbar_init(bar(BAR_KSF + s), 1); mbar_init(bar(BAR_MR + s), 4);
         }
-        mbar_init(bar(BAR_SF), 1); mbar_init(bar(BAR_SFREE), NSW);
-        mbar_init(bar(BAR_PF), NSW); mbar_init(bar(BAR_PV), 1); mbar_init(bar(BAR_QT), NSW);
-        mbar_init(bar(BAR_KSF), 1); mbar_init(bar(BAR_KSF + 1), 1);
+        mbar_init(bar(BAR_QT), NSW);
         fence_barrier_init();
         *abort_flag = status_now != 0 ? 2 : 0;
     }
-    if (warp == W_MMA) { tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS); tmem_relinquish(); }
-    if (warp == W_TMA && lane == 0) { tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_k); tma_prefetch_desc(&tmap_v); }
+    if (warp == W_QK) { tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS); tmem_relinquish(); }
+    if (warp == W_PV && lane == 0) { tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_k); tma_prefetch_desc(&tmap_v); }
     for (int i = tid; i < STAGES * 128; i += THREADS) {           // ones rows under every V^T stage
         const int st = i / 128, off = (i % 128) * 16;
         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};"
@@ -156,86 +189,89 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
 
     if (dead) {
         // fall through to the common exit
-    } else if (warp == W_TMA) {
-        // ------------------------------------------------------------------ TMA producer
+    } else if (warp == W_QK) {
+        // ------------------------------------------------------------------ Q and K loads, issuer of S = Q K^T
         if (lane == 0) {
+            constexpr uint32_t idesc_s = umma_idesc_bf16(128, BC);
+            const uint32_t q_lo = umma_desc_lo(q_s), k_lo = umma_desc_lo(k_s);
+            auto load_k = [&](int jt) {                       // K tile jt into stage jt % 2; its bytes count on QKGO
+                const int st = jt & 1;
+                mbar_expect_tx(bar(BAR_QKGO + st), K_STAGE);
+#pragma unroll
+                for (int s = 0; s < QSUB; ++s)
+                    tma_load_3d(k_s + st * K_STAGE + s * K_SUB, &tmap_k, bar(BAR_QKGO + st), 64 * s, jt * BC, bh_kv);
+            };
             mbar_expect_tx(bar(BAR_Q), Q_BYTES);
 #pragma unroll
             for (int s = 0; s < QSUB; ++s) tma_load_3d(q_s + s * 16384, &tmap_q, bar(BAR_Q), 64 * s, q0, bh_q);
-            for (int jt = 0; jt < n_tiles; ++jt) {
+            load_k(0);
+            if (n_tiles > 1) load_k(1);
+            bool ok = wait64(bar(C::Q_IN_TMEM ? BAR_QT : BAR_Q), 0, abort_flag);
+            if (!ok) fail(3);
+            for (int jt = 0; ok && jt < n_tiles; ++jt) {      // S(jt): K tile landed, S(jt-1) in registers
                 const int st = jt & 1;
                 const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
-                const int j0 = jt * BC;
-                if (!wait64(bar(BAR_KE + st), ph ^ 1u, abort_flag)) { fail(1); break; }
-                mbar_expect_tx(bar(BAR_KF + st), K_STAGE);
+                if (!wait64(bar(BAR_QKGO + st), ph, abort_flag)) { fail(4); break; }
+                tc_fence_after();
+                const uint32_t b0 = k_lo + st * (K_STAGE >> 4);
 #pragma unroll
-                for (int s = 0; s < QSUB; ++s)
-                    tma_load_3d(k_s + st * K_STAGE + s * K_SUB, &tmap_k, bar(BAR_KF + st), 64 * s, j0, bh_kv);
-                if (!wait64(bar(BAR_VE + st), ph ^ 1u, abort_flag)) { fail(2); break; }
-                mbar_expect_tx(bar(BAR_VF + st), D * 128);
-                tma_load_3d(v_s + st * V_STAGE, &tmap_v, bar(BAR_VF + st), j0, 0, bh_kv);
+                for (int kk = 0; kk < D / 16; ++kk) {          // D / 16 steps of 16 channels
+                    const uint32_t kb = b0 + (kk >> 2) * (K_SUB >> 4) + (kk & 3) * 2;
+                    if constexpr (C::Q_IN_TMEM) umma_bf16_ts_lo(tmem + S_COL, tmem + QT_COL + kk * 8, kb, idesc_s, kk ? 1u : 0u);
+                    else umma_bf16_ss_lo(tmem + S_COL, q_lo + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2, kb, idesc_s, kk ? 1u : 0u);
+                }
+                umma_commit(bar(BAR_SF + st));
+                umma_commit(bar(BAR_KE + st));
+                if (jt + 2 < n_tiles) {                        // refill the stage once this MMA has read it
+                    if (!wait_idle(bar(BAR_KE + st), ph, abort_flag)) { fail(1); break; }
+                    load_k(jt + 2);
+                }
+            }
+        }
+    } else if (warp == W_PV) {
+        // ------------------------------------------------------------------ V^T loads, issuer of [O | l] += P-hat [V | 1]
+        if (lane == 0) {
+            constexpr uint32_t idesc_o = umma_idesc_bf16(128, D == 256 ? 256 : O_COLS);
+            constexpr uint32_t idesc_l = umma_idesc_bf16(128, 16);
+            const uint32_t v_lo = umma_desc_lo(v_s);
+            auto load_v = [&](int jt) {                       // V^T tile jt into stage jt % 2; its bytes count on PVGO
+                const int st = jt & 1;
+                mbar_expect_tx(bar(BAR_PVGO + st), D * 128);
+                tma_load_3d(v_s + st * V_STAGE, &tmap_v, bar(BAR_PVGO + st), jt * BC, 0, bh_kv);
                 if (QM) {
                     // Q-Mean: the 64 channel sums of this tile's keys; their stage is free with the V stage
                     // (PV(jt-2) complete means every softmax warp is past tile jt-2)
                     mbar_expect_tx(bar(BAR_KSF + st), 256);
-                    bulk_load(smem_base + C::KSUM_OFF + st * 256, args.k_sum + (size_t)bh_kv * N + j0, 256, bar(BAR_KSF + st));
+                    bulk_load(smem_base + C::KSUM_OFF + st * 256, args.k_sum + (size_t)bh_kv * N + jt * BC, 256, bar(BAR_KSF + st));
                 }
-            }
-        }
-    } else if (warp == W_MMA) {
-        // ------------------------------------------------------------------ tcgen05 issuer
-        constexpr uint32_t idesc_s = umma_idesc_bf16(128, BC);
-        constexpr uint32_t idesc_o = umma_idesc_bf16(128, D == 256 ? 256 : O_COLS);
-        constexpr uint32_t idesc_l = umma_idesc_bf16(128, 16);
-        const uint32_t tm = __shfl_sync(0xffffffffu, tmem, 0);
-        const uint32_t q_lo = umma_desc_lo(q_s), k_lo = umma_desc_lo(k_s), v_lo = umma_desc_lo(v_s);
-        const bool leader = elect_one();
-        bool ok = true;
-        auto issue_qk = [&](int jt) {                     // S(jt) from K stage jt % 2 (D / 16 steps of 16 channels)
-            const uint32_t b0 = k_lo + (jt & 1) * (K_STAGE >> 4);
-            if (leader) {
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t kb = b0 + (kk >> 2) * (K_SUB >> 4) + (kk & 3) * 2;
-                    if constexpr (C::Q_IN_TMEM) umma_bf16_ts_lo(tm + S_COL, tm + QT_COL + kk * 8, kb, idesc_s, kk ? 1u : 0u);
-                    else umma_bf16_ss_lo(tm + S_COL, q_lo + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2, kb, idesc_s, kk ? 1u : 0u);
-                }
-                umma_commit(bar(BAR_SF));
-                umma_commit(bar(BAR_KE + (jt & 1)));
-            }
-            __syncwarp();
-        };
-        ok = wait64(bar(C::Q_IN_TMEM ? BAR_QT : BAR_Q), 0, abort_flag) && wait64(bar(BAR_KF), 0, abort_flag);
-        if (ok) { tc_fence_after(); issue_qk(0); } else if (leader) fail(3);
-        for (int jt = 0; ok && jt < n_tiles; ++jt) {
-            const int st = jt & 1;
-            const uint32_t ph = (uint32_t)(jt >> 1) & 1u, par = (uint32_t)jt & 1u;
-            if (jt + 1 < n_tiles) {                       // S(jt+1) as soon as S(jt) sits in registers
-                if (!wait64(bar(BAR_KF + (st ^ 1)), (uint32_t)((jt + 1) >> 1) & 1u, abort_flag)) { if (leader) fail(4); break; }
-                if (!wait64(bar(BAR_SFREE), par, abort_flag)) { if (leader) fail(5); break; }
+            };
+            load_v(0);
+            if (n_tiles > 1) load_v(1);
+            for (int jt = 0; jt < n_tiles; ++jt) {            // V^T tile landed, P-hat(jt) stored, history rescaled
+                const int st = jt & 1;
+                const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
+                if (!wait64(bar(BAR_PVGO + st), ph, abort_flag)) { fail(7); break; }
                 tc_fence_after();
-                issue_qk(jt + 1);
-            }
-            if (!wait64(bar(BAR_VF + st), ph, abort_flag)) { if (leader) fail(6); break; }
-            if (!wait64(bar(BAR_PF), par, abort_flag)) { if (leader) fail(7); break; }
-            tc_fence_after();
-            const uint32_t b0 = v_lo + st * (V_STAGE >> 4);
-            const uint32_t acc0 = jt > 0 ? 1u : 0u;
-            if (leader) {
+                const uint32_t b0 = v_lo + st * (V_STAGE >> 4);
+                const uint32_t acc0 = jt > 0 ? 1u : 0u;
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {            // 16 keys per step; channels (+ ones block)
-                    umma_bf16_ts_lo(tm, tm + P_COL + kk * 8, b0 + kk * 2, idesc_o, kk ? 1u : acc0);
-                    if constexpr (D == 256)                  // N = 272 does not exist: the ones block separately
-                        umma_bf16_ts_lo(tm + 256, tm + P_COL + kk * 8, b0 + ((D * 128) >> 4) + kk * 2, idesc_l, kk ? 1u : acc0);
+                for (int kk = 0; kk < 4; ++kk) {                // 16 keys per step; channels (+ ones block)
+                    umma_bf16_ts_lo(tmem, tmem + P_COL + kk * 8, b0 + kk * 2, idesc_o, kk ? 1u : acc0);
+                    if constexpr (D == 256)                      // N = 272 does not exist: the ones block separately
+                        umma_bf16_ts_lo(tmem + 256, tmem + P_COL + kk * 8, b0 + ((D * 128) >> 4) + kk * 2, idesc_l, kk ? 1u : acc0);
                 }
-                umma_commit(bar(BAR_PV));
+                umma_commit(bar(BAR_PV + st));
                 umma_commit(bar(BAR_VE + st));
+                if (jt + 2 < n_tiles) {                        // refill the stage once this MMA has read it
+                    if (!wait_idle(bar(BAR_VE + st), ph, abort_flag)) { fail(2); break; }
+                    load_v(jt + 2);
+                }
             }
-            __syncwarp();
         }
     } else {
         // ------------------------------------------------------------------ softmax / quantize
-        const int kq = warp >> 2, quarter = warp & 3;             // key half, row quarter
+        const int grp = warp >> 2, quarter = warp & 3;            // tile parity owned, row quarter
+        const int kq = grp;                                       // channel half in the Q-hat copy and in the epilogue
         const int r_loc = quarter * 32 + lane;                    // row inside the tile = TMEM lane
         const int row = q0 + r_loc;
         const uint32_t t_lane = tmem + ((uint32_t)(quarter * 32) << 16);
@@ -247,6 +283,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 if (args.dbg.blocks[3 * i] == b && args.dbg.blocks[3 * i + 1] == h && args.dbg.blocks[3 * i + 2] == qt)
                     dbg_slot = i;
         const float mu_row = (QM && row < N) ? args.q_mu[(size_t)bh_q * N + row] : 0.f;
+        float* mx_s = reinterpret_cast<float*>(smem_gen + C::MX_OFF);   // [2][128]
         float m_run = -INFINITY;
         bool ok = true;
 
@@ -254,123 +291,96 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         // channels of its row = 64 columns of packed BF16 pairs.  (d = 128: the issuer waits for the
         // Q load itself.)
         if constexpr (C::Q_IN_TMEM) {
-            static_assert(!C::Q_IN_TMEM || KS == 2 || KS == 4, "the Q copy splits a row over two or four threads");
             if (wait64(bar(BAR_Q), 0, abort_flag)) {
                 const int sw = r_loc & 7;
-                constexpr int PARTS = 4 / KS;                          // pieces of 64 channels (8 chunks, 32 columns)
 #pragma unroll
-                for (int half = 0; half < PARTS; ++half) {
+                for (int half = 0; half < 2; ++half) {             // pieces of 64 channels (8 chunks, 32 columns)
                     uint32_t qw[32];
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
-                        const int chunk = (kq * PARTS + half) * 8 + c; // 16-byte chunk of the 512-byte row
+                        const int chunk = (kq * 2 + half) * 8 + c;     // 16-byte chunk of the 512-byte row
                         const uint32_t a = q_s + (chunk >> 3) * 16384 + (r_loc >> 3) * 1024 + sw * 128 + (((chunk & 7) ^ sw) << 4);
                         asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
                                      : "=r"(qw[4 * c]), "=r"(qw[4 * c + 1]), "=r"(qw[4 * c + 2]), "=r"(qw[4 * c + 3]) : "r"(a));
                     }
-                    tmem_st32(t_lane + QT_COL + (kq * PARTS + half) * 32, qw);
+                    tmem_st32(t_lane + QT_COL + (kq * 2 + half) * 32, qw);
                 }
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar(BAR_QT));
+                arrive_lane0(bar(BAR_QT), lane);
             } else { fail(13); ok = false; }
         }
+        if (grp == 0) arrive_lane0(bar(BAR_QKGO), lane);          // S is free for tile 0
 
-        bool sf_ready = false;
-        for (int jt = 0; ok && jt < n_tiles; ++jt) {
+        for (int jt = grp; ok && jt < n_tiles; jt += 2) {
             const int j0 = jt * BC;
-            const uint32_t par = (uint32_t)jt & 1u;
-            const int kbase = j0 + kq * KPT;
-            // the poll for S(jt) was issued before the tail of the previous tile (a poll takes > 100 clk)
-            if (!sf_ready && !wait64(bar(BAR_SF), par, abort_flag)) { fail(8); ok = false; break; }
+            const int st = jt & 1;                                 // = grp
+            const uint32_t ph = (uint32_t)(jt >> 1) & 1u;          // phase parity of this group's barriers
+            if (!wait64(bar(BAR_SF + st), ph, abort_flag)) { fail(8); ok = false; break; }
             tc_fence_after();
-            // The thread pulls its own KPT scores and, for the row maximum (line 7), the rest of the row
-            // as well: the tile is one 64-key group, so row maximum = group maximum, and reading the other
-            // columns again costs less than an exchange with the other threads of the row.
-            float p[KPT], po[BC - KPT + 1];
+            float p[BC];
             {
-                uint32_t r[KPT], ro[BC - KPT + 1];
-                if constexpr (KS == 1) {
-                    uint32_t r1[32];
-                    tmem_ld32(t_lane + S_COL, reinterpret_cast<uint32_t(&)[32]>(r[0]));
-                    tmem_ld32(t_lane + S_COL + 32, r1);
-                    tmem_wait_ld();
+                uint32_t r[BC];
+                tmem_ld32(t_lane + S_COL, reinterpret_cast<uint32_t(&)[32]>(r[0]));
+                tmem_ld32(t_lane + S_COL + 32, reinterpret_cast<uint32_t(&)[32]>(r[32]));
+                tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) r[32 + i] = r1[i];
-                } else if constexpr (KS == 2) {
-                    tmem_ld32(t_lane + S_COL + kq * KPT, reinterpret_cast<uint32_t(&)[32]>(r[0]));
-                    tmem_ld32(t_lane + S_COL + (kq ^ 1) * KPT, reinterpret_cast<uint32_t(&)[32]>(ro[0]));
-                    tmem_wait_ld();
-                } else {
-                    static_assert(KS == 4, "key split of one, two or four threads per row");
-                    tmem_ld16(t_lane + S_COL + kq * KPT, reinterpret_cast<uint32_t(&)[16]>(r[0]));
-#pragma unroll
-                    for (int o = 1; o < KS; ++o)               // part kq ^ o of the row goes to ro[(o - 1) * KPT ..]
-                        tmem_ld16(t_lane + S_COL + (kq ^ o) * KPT, reinterpret_cast<uint32_t(&)[16]>(ro[(o - 1) * KPT]));
-                    tmem_wait_ld();
-                }
-#pragma unroll
-                for (int i = 0; i < KPT; ++i) p[i] = __uint_as_float(r[i]);
-#pragma unroll
-                for (int i = 0; i < BC - KPT; ++i) po[i] = __uint_as_float(ro[i]);
+                for (int i = 0; i < BC; ++i) p[i] = __uint_as_float(r[i]);
             }
             tc_fence_before();                                 // S(jt) is in registers: S(jt+1) may overwrite it
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_SFREE));
+            if (jt + 1 < n_tiles) arrive_lane0(bar(BAR_QKGO + (st ^ 1)), lane);
 
-            auto obase = [&](int o) { return j0 + (kq ^ o) * KPT; };   // first key of the o-th other part of the row
             if (QM) {                                          // Q-Mean correction (line 6): + mu_i * sum_c k~_jc
-                if (!wait64(bar(BAR_KSF + (jt & 1)), (uint32_t)(jt >> 1) & 1u, abort_flag)) { fail(15); ok = false; break; }
-                const uint32_t ks_s = smem_base + C::KSUM_OFF + (jt & 1) * 256;
-                auto add_part = [&](float* dst, int part) {     // keys part * KPT .. of the tile
+                if (!wait64(bar(BAR_KSF + st), ph, abort_flag)) { fail(15); ok = false; break; }
+                const uint32_t ks_s = smem_base + C::KSUM_OFF + st * 256;
 #pragma unroll
-                    for (int i = 0; i < KPT / 4; ++i) {
-                        float4 ks;
-                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                                     : "=f"(ks.x), "=f"(ks.y), "=f"(ks.z), "=f"(ks.w) : "r"(ks_s + (part * KPT + 4 * i) * 4));
-                        dst[4 * i] = fmaf(mu_row, ks.x, dst[4 * i]);
-                        dst[4 * i + 1] = fmaf(mu_row, ks.y, dst[4 * i + 1]);
-                        dst[4 * i + 2] = fmaf(mu_row, ks.z, dst[4 * i + 2]);
-                        dst[4 * i + 3] = fmaf(mu_row, ks.w, dst[4 * i + 3]);
-                    }
-                };
-                add_part(p, kq);
-#pragma unroll
-                for (int o = 1; o < KS; ++o) add_part(po + (o - 1) * KPT, kq ^ o);
+                for (int i = 0; i < BC / 4; ++i) {
+                    float4 ks;
+                    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                 : "=f"(ks.x), "=f"(ks.y), "=f"(ks.z), "=f"(ks.w) : "r"(ks_s + 16 * i));
+                    p[4 * i] = fmaf(mu_row, ks.x, p[4 * i]);
+                    p[4 * i + 1] = fmaf(mu_row, ks.y, p[4 * i + 1]);
+                    p[4 * i + 2] = fmaf(mu_row, ks.z, p[4 * i + 2]);
+                    p[4 * i + 3] = fmaf(mu_row, ks.w, p[4 * i + 3]);
+                }
             }
-            const bool need_mask = (args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N);
-            if (need_mask) {                                   // masked scores become -inf: exp gives exact zeros
+            if ((args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N)) {   // masked scores become -inf: exp gives exact zeros
 #pragma unroll
-                for (int i = 0; i < KPT; ++i) p[i] = (kbase + i > key_lim) ? -INFINITY : p[i];
-#pragma unroll
-                for (int o = 1; o < KS; ++o)
-#pragma unroll
-                    for (int i = 0; i < KPT; ++i)
-                        po[(o - 1) * KPT + i] = (obase(o) + i > key_lim) ? -INFINITY : po[(o - 1) * KPT + i];
+                for (int i = 0; i < BC; ++i) p[i] = (j0 + i > key_lim) ? -INFINITY : p[i];
             }
+            // row maximum = maximum of the tile's single 64-key group: eight chains of eight values
+            // (three-input maxima), then one chain over the eight
             float mx;
             {
-                float t4[KPT / 4];
+                float t8[8];
 #pragma unroll
-                for (int i = 0; i < KPT / 4; ++i) t4[i] = fmaxf(max3(p[4 * i], p[4 * i + 1], p[4 * i + 2]), p[4 * i + 3]);
-                if constexpr (KS > 1) {
-#pragma unroll
-                    for (int i = 0; i < (BC - KPT) / 4; ++i) {
-                        float& t = t4[i % (KPT / 4)];
-                        t = fmaxf(max3(t, po[4 * i], po[4 * i + 1]), fmaxf(po[4 * i + 2], po[4 * i + 3]));
-                    }
+                for (int c = 0; c < 8; ++c) {
+                    float t = max3(p[8 * c], p[8 * c + 1], p[8 * c + 2]);
+                    t = max3(t, p[8 * c + 3], p[8 * c + 4]);
+                    t = max3(t, p[8 * c + 5], p[8 * c + 6]);
+                    t8[c] = fmaxf(t, p[8 * c + 7]);
                 }
-#pragma unroll
-                for (int w = KPT / 8; w >= 1; w >>= 1)
-#pragma unroll
-                    for (int i = 0; i < w; ++i) t4[i] = fmaxf(t4[i], t4[i + w]);
-                mx = t4[0];
+                mx = max3(t8[0], t8[1], t8[2]);
+                mx = max3(mx, t8[3], t8[4]);
+                mx = max3(mx, t8[5], t8[6]);
+                mx = fmaxf(mx, t8[7]);
             }
-
+            // running maximum after the previous tile, from its owner (the other group)
+            if (jt > 0) {
+                if (!wait64(bar(BAR_MR + (st ^ 1)), (uint32_t)((jt - 1) >> 1) & 1u, abort_flag)) { fail(12); ok = false; break; }
+                m_run = mx_s[(st ^ 1) * 128 + r_loc];
+            }
+            // running maximum and rescale factor (lines 7-8), both FP16 values.  No branch: r = 1 exactly
+            // when the maximum did not move; at jt = 0 (m = -inf) r = 0 is never applied.
             const float m_new = fmaxf(m_run, f16_round(mx * args.c0));
-            float rsc = 1.f;
-            if (jt > 0 && m_new != m_run) rsc = f16_round(ex2_approx((m_run - m_new) * LOG2E));
+            if (jt + 1 < n_tiles) {                            // hand it to the owner of the next tile
+                mx_s[st * 128 + r_loc] = m_new;
+                __syncwarp();
+                arrive_lane0(bar(BAR_MR + st), lane);
+            }
+            const float rsc = f16_round(ex2_approx((m_run - m_new) * LOG2E));
             m_run = m_new;
             const float mL = m_run * LOG2E;
             const float A = p_of_score<PF32>(mx, args.c1, mL); // = max of P over the group (monotone map)
@@ -378,71 +388,25 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             // P = exp(S - m) in FP16 (line 9), P-hat = HIF4(P) (line 10)
             uint8_t* dc = nullptr;
             float* ds = nullptr;
-            if (DBG && dbg_slot >= 0 && row < N && kbase < N) {
+            if (DBG && dbg_slot >= 0 && row < N && j0 < N) {
                 const size_t r_idx = (size_t)dbg_slot * 128 + r_loc;
-                if (args.dbg.p_codes) dc = args.dbg.p_codes + r_idx * N + kbase;
-                if (args.dbg.p_step) ds = args.dbg.p_step + r_idx * (N / 4) + kbase / 4;
+                if (args.dbg.p_codes) dc = args.dbg.p_codes + r_idx * N + j0;
+                if (args.dbg.p_step) ds = args.dbg.p_step + r_idx * (N / 4) + j0 / 4;
             }
-            // poll for PV(jt-1) now, look at the answer after the exponentials
-            const bool pv_ready = jt > 0 ? mbar_test_wait(bar(BAR_PV), par ^ 1u) : true;
             uint32_t w[NU * 4];
             const PQuantConst qc = p_quant_const(args.c1, mL, A);
             exp_quantize_units<NU, 0, NU, DBG, PF32>(p, qc, A == 0.f, w, dc, ds);
-            // the P-hat columns and [O | l] are free once PV(jt-1) has completed (every warp observes
-            // every phase of that barrier, in order)
+            // the P-hat columns and [O | l] are free once P V of the previous tile has completed
             if (jt > 0) {
-                if (!pv_ready && !wait64(bar(BAR_PV), par ^ 1u, abort_flag)) { fail(10); ok = false; break; }
+                if (!wait64(bar(BAR_PV + (st ^ 1)), (uint32_t)((jt - 1) >> 1) & 1u, abort_flag)) { fail(10); ok = false; break; }
                 tc_fence_after();
             }
-            sf_ready = mbar_test_wait(bar(BAR_SF), par ^ 1u);   // S(jt+1): answer used at the top of the next tile
-            if constexpr (NU == 8) tmem_st32(t_lane + P_COL, w);
-            else if constexpr (NU == 4) tmem_st16(t_lane + P_COL + kq * (KPT / 2), w);
-            else tmem_st8(t_lane + P_COL + kq * (KPT / 2), w);
-            // rescale history (line 8): each half of the row's threads owns half of the d + 16 columns
-            if constexpr (D == 128 && KS == 2) {            // all of the thread's 72 columns in one round trip
-                if (__any_sync(0xffffffffu, rsc != 1.f)) {
-                    const uint32_t t_o = t_lane + kq * 72;
-                    const uint64_t rr = pack2(rsc, rsc);
-                    uint32_t r0[32], r1[32], r2[4], r3[4];
-                    tmem_ld32(t_o, r0);
-                    tmem_ld32(t_o + 32, r1);
-                    tmem_ld4(t_o + 64, r2);
-                    tmem_ld4(t_o + 68, r3);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float x0, x1;
-                        unpack2(mul2(pack2(__uint_as_float(r0[i]), __uint_as_float(r0[i + 1])), rr), x0, x1);
-                        r0[i] = __float_as_uint(x0);
-                        r0[i + 1] = __float_as_uint(x1);
-                    }
-                    tmem_st32(t_o, r0);
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float x0, x1;
-                        unpack2(mul2(pack2(__uint_as_float(r1[i]), __uint_as_float(r1[i + 1])), rr), x0, x1);
-                        r1[i] = __float_as_uint(x0);
-                        r1[i + 1] = __float_as_uint(x1);
-                    }
-                    tmem_st32(t_o + 32, r1);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        r2[i] = __float_as_uint(__uint_as_float(r2[i]) * rsc);
-                        r3[i] = __float_as_uint(__uint_as_float(r3[i]) * rsc);
-                    }
-                    tmem_st4(t_o + 64, r2);
-                    tmem_st4(t_o + 68, r3);
-                }
-            } else
-            if (__any_sync(0xffffffffu, rsc != 1.f)) {
-                constexpr int CW = O_COLS / KS;                // 136 or 72
-                const uint32_t t_o = t_lane + kq * CW;
+            tmem_st32(t_lane + P_COL, w);
+            // rescale of the history (line 8): the d channels and the normaliser column (the other columns of
+            // the ones block are never read)
+            if (jt > 0 && __any_sync(0xffffffffu, rsc != 1.f)) {
                 const uint64_t rr = pack2(rsc, rsc);
-#pragma unroll
-                for (int cc = 0; cc < CW / 32; ++cc) {
-                    uint32_t r[32];
-                    tmem_ld32(t_o + cc * 32, r);
-                    tmem_wait_ld();
+                auto scale32 = [&](uint32_t (&r)[32]) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
                         float x0, x1;
@@ -450,35 +414,31 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                         r[i] = __float_as_uint(x0);
                         r[i + 1] = __float_as_uint(x1);
                     }
-                    tmem_st32(t_o + cc * 32, r);
-                }
+                };
+                uint32_t rl[1];
+                tmem_ld1(t_lane + D, rl);
 #pragma unroll
-                if constexpr (CW % 32 == 16) {                 // 144 = 4 x 32 + 16: only the l column of the tail matters
-                    uint32_t r[4];
-                    tmem_ld4(t_o + (CW / 32) * 32, r);
+                for (int cc = 0; cc < D / 64; ++cc) {          // 64 columns per round trip
+                    uint32_t r0[32], r1[32];
+                    tmem_ld32(t_lane + cc * 64, r0);
+                    tmem_ld32(t_lane + cc * 64 + 32, r1);
                     tmem_wait_ld();
-                    r[0] = __float_as_uint(__uint_as_float(r[0]) * rsc);
-                    tmem_st4(t_o + (CW / 32) * 32, r);
-                } else {
-#pragma unroll
-                    for (int cc = 0; cc < (CW % 32) / 4; ++cc) {
-                        uint32_t r[4];
-                        tmem_ld4(t_o + (CW / 32) * 32 + cc * 4, r);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * rsc);
-                        tmem_st4(t_o + (CW / 32) * 32 + cc * 4, r);
-                    }
+                    scale32(r0);
+                    tmem_st32(t_lane + cc * 64, r0);
+                    scale32(r1);
+                    tmem_st32(t_lane + cc * 64 + 32, r1);
                 }
+                rl[0] = __float_as_uint(__uint_as_float(rl[0]) * rsc);
+                tmem_st1(t_lane + D, rl);
             }
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar(BAR_PF));
+            arrive_lane0(bar(BAR_PVGO + st), lane);
         }
 
         // finalize: out = O / l with l rounded to FP16 (line 13); half kq writes channels (d/2)*kq..
-        if (ok && wait64(bar(BAR_PV), (uint32_t)(n_tiles - 1) & 1u, abort_flag)) {
+        if (ok && wait64(bar(BAR_PV + ((n_tiles - 1) & 1)), (uint32_t)((n_tiles - 1) >> 1) & 1u, abort_flag)) {
             tc_fence_after();
             uint32_t lr[4];
             tmem_ld4(t_lane + D, lr);
@@ -489,19 +449,19 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             // q = fma(fma(-q0, l, O), y, q0) (Markstein's correction step; no value here is near the ends of
             // the FP32 range: l >= 2^-24 is an FP16 value and |O| <= l * max|V|)
             const float rl = __frcp_rn(l16);
-            if (DBG && dbg_slot >= 0 && row < N && kq == 0) {
+            if (DBG && dbg_slot >= 0 && row < N && grp == ((n_tiles - 1) & 1)) {   // the owner of the last tile
                 if (args.dbg.l_out) args.dbg.l_out[dbg_slot * 128 + r_loc] = ell;
                 if (args.dbg.m_out) args.dbg.m_out[dbg_slot * 128 + r_loc] = m_run;
             }
-            const size_t orow = ((size_t)bh_q * N + row) * D + kq * (D / KS);
+            const size_t orow = ((size_t)bh_q * N + row) * D + kq * (D / 2);
             // FP32 output goes through a 32 x 32 transpose in shared memory (the K stages are idle by now:
             // every load has landed and every MMA has completed), so that a warp stores four whole
             // 128-byte lines per instruction instead of 32 pieces of 16 bytes.
             const uint32_t stage = k_s + (uint32_t)warp * 4096u;
 #pragma unroll
-            for (int cc = 0; cc < D / KS / 32; ++cc) {
+            for (int cc = 0; cc < D / 2 / 32; ++cc) {
                 uint32_t r[32];
-                tmem_ld32(t_lane + kq * (D / KS) + cc * 32, r);
+                tmem_ld32(t_lane + kq * (D / 2) + cc * 32, r);
                 tmem_wait_ld();
                 float o[32];
 #pragma unroll
@@ -519,7 +479,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                     __syncwarp();
                     const int c4 = lane & 7;
                     float* obase = reinterpret_cast<float*>(args.out) + ((size_t)bh_q * N + q0 + quarter * 32) * D +
-                                   kq * (D / KS) + cc * 32 + c4 * 4;
+                                   kq * (D / 2) + cc * 32 + c4 * 4;
 #pragma unroll
                     for (int it = 0; it < 8; ++it) {
                         const int rr = it * 4 + (lane >> 3);
@@ -554,7 +514,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
 
     tc_fence_before();
     __syncthreads();
-    if (warp == W_MMA) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
+    if (warp == W_QK) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
 }
 
 template <int DH, bool DBG, bool PF32, bool QM>
