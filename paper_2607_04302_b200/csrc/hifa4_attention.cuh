@@ -239,9 +239,10 @@ __device__ __forceinline__ void exp_quantize_units(const float (&acc)[NU * 8], c
             y[i] = add2(mul2_rz(pack2(p[i], p[4 + i]), k.inv44), mm);
             unpack2(fma2(y[i], k.s44, cc), v[i], v[4 + i]);
         }
+        // BF16 image: every value has at most 8 significant bits, so the upper halves of the FP32 patterns
+        // are the BF16 values (a byte permute instead of a conversion)
 #pragma unroll
-        for (int i = 0; i < 4; ++i)
-            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[4 * u + i]) : "f"(v[2 * i + 1]), "f"(v[2 * i]));
+        for (int i = 0; i < 4; ++i) w[4 * u + i] = __byte_perm(__float_as_uint(v[2 * i]), __float_as_uint(v[2 * i + 1]), 0x7632);
         if (DBG) {
             float c[8];
 #pragma unroll
