@@ -145,11 +145,33 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     const int last_key = args.causal ? min(q0 + 127, N - 1) : N - 1;
     const int n_tiles = last_key / BC + 1;
 
-    if (tid == 0) {
+    // TMA loads; the bytes of a K tile count on the barrier that releases its S = Q K^T, those of a V^T tile
+    // on the barrier that releases its P V (one thread of warp W_QK resp. W_PV calls these)
+    auto load_k = [&](int jt) {                               // K tile jt into stage jt % 2
+        const int st = jt & 1;
+        mbar_expect_tx(bar(BAR_QKGO + st), K_STAGE);
+#pragma unroll
+        for (int s = 0; s < QSUB; ++s)
+            tma_load_3d(k_s + st * K_STAGE + s * K_SUB, &tmap_k, bar(BAR_QKGO + st), 64 * s, jt * BC, bh_kv);
+    };
+    auto load_v = [&](int jt) {                               // V^T tile jt into stage jt % 2
+        const int st = jt & 1;
+        mbar_expect_tx(bar(BAR_PVGO + st), D * 128);
+        tma_load_3d(v_s + st * V_STAGE, &tmap_v, bar(BAR_PVGO + st), jt * BC, 0, bh_kv);
+        if (QM) {
+            // Q-Mean: the 64 channel sums of this tile's keys; their stage is free with the V stage
+            // (P V of tile jt-2 complete means every softmax warp is past tile jt-2)
+            mbar_expect_tx(bar(BAR_KSF + st), 256);
+            bulk_load(smem_base + C::KSUM_OFF + st * 256, args.k_sum + (size_t)bh_kv * N + jt * BC, 256, bar(BAR_KSF + st));
+        }
+    };
+
+    if (warp == W_QK && lane == 0) {
         // A CTA that starts after another one reported a failure does nothing.  One thread reads the status
-        // word (the load is in flight during the set-up below) and publishes the verdict through shared
-        // memory, so that all roles of the CTA agree on it.
-        const int status_now = args.d_status ? *reinterpret_cast<volatile int*>(args.d_status) : 0;
+        // word and publishes the verdict through shared memory, so that all roles of the CTA agree on it.
+        // The same thread sets the barriers up and starts the first loads at once (Q, two K tiles, two V^T
+        // tiles), so that they are in flight while the rest of the CTA sets itself up.
+        int status_now = args.d_status ? *reinterpret_cast<volatile int*>(args.d_status) : 0;
         mbar_init(bar(BAR_Q), 1);
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar(BAR_QKGO + s), 5); mbar_init(bar(BAR_KE + s), 1);
@@ -159,10 +181,22 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         }
         mbar_init(bar(BAR_QT), NSW);
         fence_barrier_init();
+        // The launch lets this grid start while its predecessor in the stream is still running; nothing the
+        // predecessor wrote is touched before this point.  A non-zero status word read before it may be one
+        // that the preceding work in the stream has cleared since: that (rare) verdict is read again.
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (status_now != 0) status_now = *reinterpret_cast<volatile int*>(args.d_status);
         *abort_flag = status_now != 0 ? 2 : 0;
+        if (status_now == 0) {
+            mbar_expect_tx(bar(BAR_Q), Q_BYTES);
+#pragma unroll
+            for (int s = 0; s < QSUB; ++s) tma_load_3d(q_s + s * 16384, &tmap_q, bar(BAR_Q), 64 * s, q0, bh_q);
+            load_k(0);
+            load_v(0);
+            if (n_tiles > 1) { load_k(1); load_v(1); }
+        }
     }
-    if (warp == W_QK) { tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS); tmem_relinquish(); }
-    if (warp == W_PV && lane == 0) { tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_k); tma_prefetch_desc(&tmap_v); }
+    if (warp == W_QK) { __syncwarp(); tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS); tmem_relinquish(); }
     for (int i = tid; i < STAGES * 128; i += THREADS) {           // ones rows under every V^T stage
         const int st = i / 128, off = (i % 128) * 16;
         asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};"
@@ -170,13 +204,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     }
     fence_proxy_async_smem();
     tc_fence_before();
-    // The launch lets this grid start while its predecessor in the stream is still running (its CTAs
-    // become resident and set themselves up as SMs drain); nothing the predecessor wrote is touched
-    // before this point.
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    // The status word was read before the wait; a non-zero value may be one that the preceding work in the
-    // stream has cleared since, so only that (rare) verdict is confirmed by a second read.
-    if (tid == 0 && *abort_flag) *abort_flag = *reinterpret_cast<volatile int*>(args.d_status) != 0 ? 2 : 0;
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
@@ -194,18 +222,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         if (lane == 0) {
             constexpr uint32_t idesc_s = umma_idesc_bf16(128, BC);
             const uint32_t q_lo = umma_desc_lo(q_s), k_lo = umma_desc_lo(k_s);
-            auto load_k = [&](int jt) {                       // K tile jt into stage jt % 2; its bytes count on QKGO
-                const int st = jt & 1;
-                mbar_expect_tx(bar(BAR_QKGO + st), K_STAGE);
-#pragma unroll
-                for (int s = 0; s < QSUB; ++s)
-                    tma_load_3d(k_s + st * K_STAGE + s * K_SUB, &tmap_k, bar(BAR_QKGO + st), 64 * s, jt * BC, bh_kv);
-            };
-            mbar_expect_tx(bar(BAR_Q), Q_BYTES);
-#pragma unroll
-            for (int s = 0; s < QSUB; ++s) tma_load_3d(q_s + s * 16384, &tmap_q, bar(BAR_Q), 64 * s, q0, bh_q);
-            load_k(0);
-            if (n_tiles > 1) load_k(1);
             bool ok = wait64(bar(C::Q_IN_TMEM ? BAR_QT : BAR_Q), 0, abort_flag);
             if (!ok) fail(3);
             for (int jt = 0; ok && jt < n_tiles; ++jt) {      // S(jt): K tile landed, S(jt-1) in registers
@@ -234,19 +250,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             constexpr uint32_t idesc_o = umma_idesc_bf16(128, D == 256 ? 256 : O_COLS);
             constexpr uint32_t idesc_l = umma_idesc_bf16(128, 16);
             const uint32_t v_lo = umma_desc_lo(v_s);
-            auto load_v = [&](int jt) {                       // V^T tile jt into stage jt % 2; its bytes count on PVGO
-                const int st = jt & 1;
-                mbar_expect_tx(bar(BAR_PVGO + st), D * 128);
-                tma_load_3d(v_s + st * V_STAGE, &tmap_v, bar(BAR_PVGO + st), jt * BC, 0, bh_kv);
-                if (QM) {
-                    // Q-Mean: the 64 channel sums of this tile's keys; their stage is free with the V stage
-                    // (PV(jt-2) complete means every softmax warp is past tile jt-2)
-                    mbar_expect_tx(bar(BAR_KSF + st), 256);
-                    bulk_load(smem_base + C::KSUM_OFF + st * 256, args.k_sum + (size_t)bh_kv * N + jt * BC, 256, bar(BAR_KSF + st));
-                }
-            };
-            load_v(0);
-            if (n_tiles > 1) load_v(1);
             for (int jt = 0; jt < n_tiles; ++jt) {            // V^T tile landed, P-hat(jt) stored, history rescaled
                 const int st = jt & 1;
                 const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
