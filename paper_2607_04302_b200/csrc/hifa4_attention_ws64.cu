@@ -169,8 +169,8 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     if (warp == W_QK && lane == 0) {
         // A CTA that starts after another one reported a failure does nothing.  One thread reads the status
         // word and publishes the verdict through shared memory, so that all roles of the CTA agree on it.
-        // The same thread sets the barriers up and starts the first loads at once (Q, two K tiles, two V^T
-        // tiles), so that they are in flight while the rest of the CTA sets itself up.
+        // The same thread sets the barriers up and starts the first loads at once (Q and two K tiles), so that
+        // they are in flight while the rest of the CTA sets itself up.
         int status_now = args.d_status ? *reinterpret_cast<volatile int*>(args.d_status) : 0;
         mbar_init(bar(BAR_Q), 1);
         for (int s = 0; s < STAGES; ++s) {
@@ -192,8 +192,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
 #pragma unroll
             for (int s = 0; s < QSUB; ++s) tma_load_3d(q_s + s * 16384, &tmap_q, bar(BAR_Q), 64 * s, q0, bh_q);
             load_k(0);
-            load_v(0);
-            if (n_tiles > 1) { load_k(1); load_v(1); }
+            if (n_tiles > 1) load_k(1);
         }
     }
     if (warp == W_QK) { __syncwarp(); tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS); tmem_relinquish(); }
@@ -250,6 +249,8 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             constexpr uint32_t idesc_o = umma_idesc_bf16(128, D == 256 ? 256 : O_COLS);
             constexpr uint32_t idesc_l = umma_idesc_bf16(128, 16);
             const uint32_t v_lo = umma_desc_lo(v_s);
+            load_v(0);
+            if (n_tiles > 1) load_v(1);
             for (int jt = 0; jt < n_tiles; ++jt) {            // V^T tile landed, P-hat(jt) stored, history rescaled
                 const int st = jt & 1;
                 const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
