@@ -205,8 +205,12 @@ static int cmp_float(const void* a, const void* b)
  * Gate").  q_cal [S][Hq][Ncal][d], k_cal [S][Hkv][Ncal][d].
  * Per sample the per-channel statistic is the maximum magnitude over tokens
  * (and, for Q, over the query heads that share the KV head); samples are
- * combined by root-mean-square.  s = Kagg^alpha / Qagg^(1-alpha).
- * mode: 0 bypass, 1 strong (alpha .5), 2 mild (.25), 3 gate decides, 4 alpha given.
+ * combined by root-mean-square (the aggregator the paper adopts) or, as the
+ * alternatives of its aggregator comparison (table "calib"), by the mean or by
+ * the 99th percentile (nearest rank) of the per-sample maxima.
+ * s = Kagg^alpha / Qagg^(1-alpha).
+ * mode: 0 bypass, 1 strong (alpha .5), 2 mild (.25), 3 gate decides, 4 alpha given;
+ * plus 0x100 for the mean aggregator, 0x200 for the 99th percentile.
  * stats[0] = rho_K = max|K| / P99(|K|) (nearest rank), stats[1] = T = max|K|/max|Q|,
  * stats[2] = branch taken (0 bypass, 1 strong, 2 mild), stats[3] = alpha used. */
 int hifa4_oracle_smooth_calibrate(const float* q_cal, const float* k_cal, int S, int Hq, int Hkv,
@@ -214,6 +218,12 @@ int hifa4_oracle_smooth_calibrate(const float* q_cal, const float* k_cal, int S,
                                   float* s, float* inv_s, double* kagg_out, double* qagg_out,
                                   double* stats)
 {
+    const int aggregator = (mode >> 8) & 3;      /* 0 RMS, 1 mean, 2 99th percentile */
+    mode &= 0xFF;
+    if (aggregator > 2) return 3;
+    double* kms = (double*)malloc(sizeof(double) * 2 * S);
+    if (!kms) return 2;
+    double* qms = kms + S;
     long nk = (long)S * Hkv * Ncal * d, nq = (long)S * Hq * Ncal * d;
     double kmaxall = 0, qmaxall = 0;
     for (long i = 0; i < nk; ++i) if (fabs(k_cal[i]) > kmaxall) kmaxall = fabs(k_cal[i]);
@@ -255,8 +265,29 @@ int hifa4_oracle_smooth_calibrate(const float* q_cal, const float* k_cal, int S,
                 }
                 ksum += km * km;
                 qsum += qm * qm;
+                kms[n] = km;
+                qms[n] = qm;
             }
             double kagg = sqrt(ksum / S), qagg = sqrt(qsum / S);
+            if (aggregator == 1) {                       /* mean of the per-sample maxima */
+                kagg = qagg = 0;
+                for (int n = 0; n < S; ++n) { kagg += kms[n]; qagg += qms[n]; }
+                kagg /= S;
+                qagg /= S;
+            } else if (aggregator == 2) {                /* nearest-rank 99th percentile of them */
+                long rank = (long)ceil(0.99 * (double)S);
+                if (rank < 1) rank = 1;
+                for (int pass = 0; pass < 2; ++pass) {   /* selection by counting: S is small */
+                    double* v = pass ? qms : kms;
+                    double pick = 0;
+                    for (int a = 0; a < S; ++a) {
+                        long below = 0, not_above = 0;
+                        for (int b2 = 0; b2 < S; ++b2) { below += v[b2] < v[a]; not_above += v[b2] <= v[a]; }
+                        if (below < rank && rank <= not_above) { pick = v[a]; break; }
+                    }
+                    if (pass) qagg = pick; else kagg = pick;
+                }
+            }
             if (kagg_out) kagg_out[g * d + c] = kagg;
             if (qagg_out) qagg_out[g * d + c] = qagg;
             double sv = 1.0;
@@ -264,6 +295,7 @@ int hifa4_oracle_smooth_calibrate(const float* q_cal, const float* k_cal, int S,
             s[g * d + c] = (float)sv;
             inv_s[g * d + c] = 1.0f / s[g * d + c];
         }
+    free(kms);
     return 0;
 }
 

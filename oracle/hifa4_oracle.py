@@ -166,9 +166,14 @@ def ksum_rows(x: np.ndarray, scale, dtype: int) -> np.ndarray:
     return ks
 
 
+AGG_RMS, AGG_MEAN, AGG_P99 = 0, 0x100, 0x200
+
+
 def smooth_calibrate(q_cal: np.ndarray, k_cal: np.ndarray, mode: int, alpha: float = 0.0,
-                     q_to_kv=None):
-    """q_cal [S,Hq,Ncal,d], k_cal [S,Hkv,Ncal,d] -> dict(s, inv_s, kagg, qagg, stats)."""
+                     q_to_kv=None, aggregator: int = AGG_RMS):
+    """q_cal [S,Hq,Ncal,d], k_cal [S,Hkv,Ncal,d] -> dict(s, inv_s, kagg, qagg, stats).
+    aggregator: how the per-sample channel maxima are combined over samples (RMS, mean, 99th percentile)."""
+    mode = int(mode) | int(aggregator)
     q_cal = np.ascontiguousarray(q_cal, np.float32)
     k_cal = np.ascontiguousarray(k_cal, np.float32)
     S, Hq, Ncal, d = q_cal.shape

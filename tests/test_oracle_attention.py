@@ -85,6 +85,32 @@ def test_smooth_qk_invariance_and_equalisation(oracle):
                           oracle.attention_rows(q, pos, k, v, one, one, **kw))
 
 
+def test_calibration_aggregators_against_numpy(oracle):
+    """The three ways of combining the per-sample channel maxima over the calibration set (the paper's
+    aggregator comparison: RMS adopted, mean and 99th percentile as alternatives), pinned against numpy
+    reductions of the per-sample maxima (np.percentile's inverted-CDF method is the nearest-rank rule)."""
+    rng = np.random.default_rng(21)
+    S, Hq, Hkv, Ncal, d = 120, 2, 1, 4, 64
+    qc = (rng.standard_normal((S, Hq, Ncal, d)) * np.exp(rng.standard_normal((S, 1, 1, 1)) * 0.4)).astype(np.float32)
+    kc = (rng.standard_normal((S, Hkv, Ncal, d)) * np.exp(rng.standard_normal((S, 1, 1, 1)) * 0.4)).astype(np.float32)
+    kmax = np.abs(kc.astype(np.float64)).max(axis=2)[:, 0]              # [S, d]
+    qmax = np.abs(qc.astype(np.float64)).max(axis=(1, 2))               # [S, d], both query heads share the KV head
+    want = {oracle.AGG_RMS: (np.sqrt((kmax ** 2).mean(0)), np.sqrt((qmax ** 2).mean(0))),
+            oracle.AGG_MEAN: (kmax.mean(0), qmax.mean(0)),
+            oracle.AGG_P99: (np.percentile(kmax, 99, axis=0, method="inverted_cdf"),
+                             np.percentile(qmax, 99, axis=0, method="inverted_cdf"))}
+    got = {}
+    for agg, (kw, qw) in want.items():
+        cal = oracle.smooth_calibrate(qc, kc, mode=2, aggregator=agg)
+        assert np.allclose(cal["kagg"][0], kw, rtol=1e-13) and np.allclose(cal["qagg"][0], qw, rtol=1e-13)
+        s_want = kw ** 0.25 / qw ** 0.75
+        assert np.allclose(cal["s"][0], s_want, rtol=1e-6) and np.array_equal(cal["inv_s"], (1.0 / cal["s"]).astype(np.float32))
+        got[agg] = cal["kagg"][0]
+    # the three differ on this data, in the order mean < RMS < 99th percentile (second largest of 120 samples)
+    assert np.all(got[oracle.AGG_MEAN] < got[oracle.AGG_RMS]) and np.all(got[oracle.AGG_RMS] < got[oracle.AGG_P99])
+    assert np.array_equal(got[oracle.AGG_P99], np.sort(kmax, axis=0)[-2])
+
+
 def test_calibration_modes_and_gate(oracle):
     rng = np.random.default_rng(5)
     qc = rng.standard_normal((3, 4, 64, 64)).astype(np.float32)
