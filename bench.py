@@ -2,8 +2,10 @@
 """Benchmark of the HiFA4 hot path on B200: one step = Smooth-QK + HIF4 quantization of Q/K/V
 followed by the fused 4-bit-operand attention forward (Algorithm 1) over one batch of synthetic
 prefill activations.  Prints ONE JSON line: metric, value (whole-job TFLOP/s over the timed steps),
-roofline (attention launch against the measured BF16 tensor peak), quantize split, end-to-end figure
-with host buffers, clocks sampled during the timed region, CPU-oracle baseline and context numbers.
+roofline (attention launch against the measured BF16 tensor peak), quantize split, end-to-end figures
+with host buffers (FP16 and FP32 output), clocks sampled during the timed region, CPU-oracle baseline,
+dense GEMM peaks measured in the same run (BF16, FP8), context numbers and a sweep over the other
+configurations and variants.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C2] [--impl ours|reference]
 
@@ -33,8 +35,15 @@ UNIT = "TFLOP/s"
 NOMINAL = {"fp4": 9000.0, "fp8": 4500.0, "bf16": 2250.0}      # dense TFLOP/s, context only
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture
 # summarised in profiles/attention_fwd_ws_C2.md (bytes per launch; None where not captured)
-NCU_INSTR_PER_WARP_SCORE = {"attention_fwd_ws64_kernel<128>": 17.9}   # profiles/attention_fwd_ws64_C2.md
+# executed warp instructions per 32 scores (ncu opcode counters) and DRAM bytes per launch, from the captures
+# summarised in profiles/attention_fwd_ws64_C2.md and profiles/attention_fwd_ws_bc128_C2.md
+NCU_INSTR_PER_WARP_SCORE = {"attention_fwd_ws64_kernel<128>": 15.5}
 NCU_TRAFFIC_BYTES = {("C2-qwen3-8b-4k", 64): 68.70e6, ("C2-qwen3-8b-4k", 128): 67.14e6}
+# Issue slots the method itself needs per score on this machine (per 32 scores one warp instruction each):
+# exponential 1, scale-subtract FMA 0.5 (packed), FP16 round trip 1.5, row maximum 0.5, subgroup maxima 0.5,
+# shift selection 1.25, scale-and-round 1.5 (packed), BF16 image 0.5, rescale of the history about 0.7,
+# per-row scalars and tensor-memory traffic about 0.6: 8.5.
+ALGORITHMIC_SLOTS_PER_SCORE = 8.5
 
 
 def attn_flops(cfg) -> float:
@@ -131,6 +140,80 @@ def whole_job_tflops(cfg, world: int, steps: int, total_ms: float) -> float:
     return world * attn_flops(cfg) * steps / (total_ms * 1e-3) / 1e12
 
 
+def measure_gemm_peaks(dev):
+    """Dense GEMM throughput measured in this run (8192^3, best of 5): BF16 through torch.matmul, FP8 (e4m3)
+    through torch._scaled_mm; FP4 only if the installed torch exposes a dense FP4 matmul (it does not: null)."""
+    res = {"bf16_tflops": None, "fp8_tflops": None, "fp4_tflops": None}
+    n = 8192
+    try:
+        a = torch.randn((n, n), device=dev, dtype=torch.bfloat16)
+        b = torch.randn((n, n), device=dev, dtype=torch.bfloat16)
+
+        def best(fn):
+            for _ in range(2):
+                fn()
+            torch.cuda.synchronize()
+            t = []
+            for _ in range(5):
+                e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+                e0.record(); fn(); e1.record()
+                torch.cuda.synchronize()
+                t.append(e0.elapsed_time(e1))
+            return 2.0 * n ** 3 / (min(t) * 1e-3) / 1e12
+
+        res["bf16_tflops"] = best(lambda: torch.matmul(a, b))
+        a8 = a.to(torch.float8_e4m3fn)
+        b8 = b.to(torch.float8_e4m3fn).t().contiguous().t()          # column-major second operand
+        one = torch.ones((), device=dev, dtype=torch.float32)
+        res["fp8_tflops"] = best(lambda: torch._scaled_mm(a8, b8, scale_a=one, scale_b=one, out_dtype=torch.bfloat16))
+    except Exception as e:                                             # context only: never fail the bench on it
+        res["error"] = str(e)[:160]
+    return res
+
+
+def time_workload(hb, cfg, dev, steps, warmup, flush_l2, s=None, inv_s=None, qmean=False, p_f32=False):
+    """Device-resident timing of one configuration: per-step time of quantize + attention (events around each
+    step, L2 flushed between steps) and, from a second pass with one more event, the attention launch alone."""
+    q, k, v = synth.make_qkv_device(cfg, dev)
+    dt = hb._DT[q.dtype]
+    qkv = hb.alloc_qkv(cfg.B, cfg.Hq, cfg.Hkv, cfg.N, cfg.d, dt, dev, qmean=qmean)
+    out = torch.empty((cfg.B, cfg.Hq, cfg.N, cfg.d), dtype=torch.float32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def step(split):
+        hb.quantize_qkv(q, k, v, s, inv_s, out=qkv, d_status=status, qmean=qmean)
+        mid = None
+        if split:
+            mid = torch.cuda.Event(enable_timing=True)
+            mid.record()
+        hb.attention_fwd(qkv, cfg.causal, Bc=cfg.Bc, out_dtype=hb.F32, out=out, d_status=status,
+                         p_dtype=hb.F32 if p_f32 else hb.F16, qmean=qmean)
+        return mid
+
+    for _ in range(warmup):
+        flush_l2(); step(False)
+    torch.cuda.synchronize()
+    ev, ev2 = [], []
+    for _ in range(steps):
+        flush_l2()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record(); step(False); b.record()
+        ev.append((a, b))
+    for _ in range(steps):
+        flush_l2()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record(); m = step(True); b.record()
+        ev2.append((a, m, b))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, f"device status {int(status.item())}"
+    ms = sum(a.elapsed_time(b) for a, b in ev) / steps
+    attn = sum(m.elapsed_time(b) for _, m, b in ev2) / steps
+    quant = sum(a.elapsed_time(m) for a, m, _ in ev2) / steps
+    fl = attn_flops(cfg)
+    return {"ms_per_step": ms, "tflops": fl / (ms * 1e-3) / 1e12, "attention_ms": attn,
+            "attention_tflops": fl / (attn * 1e-3) / 1e12, "quantize_ms": quant}
+
+
 def oracle_time(cfg, q, k, v, s, inv_s, heads):
     """Time the CPU oracle, as it stands, on whole heads of the workload (batch 0)."""
     from oracle import hifa4_oracle as orc
@@ -212,6 +295,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-context", action="store_true", help="skip the torch SDPA / N=8192 context numbers")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="skip the sweep over the other configurations and variants (headline workload only)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -346,34 +431,22 @@ def main():
     total_ms = max_over_ranks(dist, total_ms, dev)
     assert int(status.item()) == 0, f"device status {int(status.item())}"
 
-    # ---- end to end through the raw C-ABI entry point with host buffers (pinned), copies timed
-    e2e = None
+    # ---- end to end through the raw C-ABI entry point with host buffers (pinned), copies timed.  Two figures:
+    # FP16 output (the method's final normalisation is FP16: Appendix, "FP16 operations") and FP32 output (the
+    # dtype the parity tests judge); the FP16 one is the line's `e2e`.
+    e2e = e2e_f32 = None
     if not big and not args.qmean:
         pq, pk, pv = qh.pin_memory(), kh.pin_memory(), vh.pin_memory()
-        po = torch.empty(out.shape, dtype=torch.float32).pin_memory()
         dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
-        # One problem per (batch, KV head group): its Q/K/V slices are contiguous, so each goes through
+        # One problem per (batch, pair of KV head groups): its Q/K/V slices are contiguous, so each goes through
         # hifa4_attention_fwd_raw on its own, and three streams keep the host-to-device copy of one
         # slice, the kernels of another and the device-to-host copy of a third in flight together.
         G = cfg.Hq // cfg.Hkv
+        GPS = 2 if cfg.Hkv % 2 == 0 else 1                               # KV head groups per slice
         streams = [torch.cuda.Stream(device=dev) for _ in range(3)]
-        ws_bytes = hb.attention_raw_workspace_bytes(1, G, 1, cfg.N, cfg.d, dt, cfg.causal, cfg.Bc)
+        ws_bytes = hb.attention_raw_workspace_bytes(1, G * GPS, GPS, cfg.N, cfg.d, dt, cfg.causal, cfg.Bc)
         ws_s = [torch.empty(ws_bytes, dtype=torch.uint8, device=dev) for _ in streams]
-        slices = [(bb, g) for bb in range(cfg.B) for g in range(cfg.Hkv)]
-
-        def e2e_step():
-            for i, (bb, g) in enumerate(slices):
-                st_i = streams[i % len(streams)]
-                hs = slice(g * G, (g + 1) * G)
-                with torch.cuda.stream(st_i):
-                    dq[bb:bb + 1, hs].copy_(pq[bb:bb + 1, hs], non_blocking=True)
-                    dk[bb:bb + 1, g:g + 1].copy_(pk[bb:bb + 1, g:g + 1], non_blocking=True)
-                    dv[bb:bb + 1, g:g + 1].copy_(pv[bb:bb + 1, g:g + 1], non_blocking=True)
-                    hb.attention_fwd_raw(dq[bb:bb + 1, hs], dk[bb:bb + 1, g:g + 1], dv[bb:bb + 1, g:g + 1],
-                                         None if s is None else s[g:g + 1], None if inv_s is None else inv_s[g:g + 1],
-                                         cfg.causal, Bc=cfg.Bc, out=out[bb:bb + 1, hs], workspace=ws_s[i % len(streams)],
-                                         d_status=status)
-                    po[bb:bb + 1, hs].copy_(out[bb:bb + 1, hs], non_blocking=True)
+        slices = [(bb, g) for bb in range(cfg.B) for g in range(0, cfg.Hkv, GPS)]
 
         def fork():
             e = torch.cuda.Event()
@@ -387,29 +460,51 @@ def main():
                 e.record(st_i)
                 torch.cuda.current_stream().wait_event(e)
 
-        fork()
-        for _ in range(3):
-            e2e_step()
-        join()
-        barrier()
-        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
-        n_e2e = max(3, min(args.steps, 10))
-        a.record()
-        fork()
-        for _ in range(n_e2e):
-            e2e_step()
-        join()
-        b.record()
-        barrier()
-        assert int(status.item()) == 0, f"device status {int(status.item())}"
-        assert torch.equal(po.to(dev), out), "end-to-end output differs from the device result"
-        e_ms = a.elapsed_time(b)
-        e_ms = max_over_ranks(dist, e_ms, dev)
-        h2d = (pq.numel() + pk.numel() + pv.numel()) * pq.element_size()
-        e2e = {"value": whole_job_tflops(cfg, world, n_e2e, e_ms), "unit": UNIT,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": po.numel() * 4, "ms_per_step": e_ms / n_e2e,
-               "how": f"hifa4_attention_fwd_raw per (batch, KV head group) slice, {len(slices)} slices over "
-                      f"{len(streams)} streams, pinned host buffers"}
+        def e2e_run(out_code, torch_dt):
+            d_out = out if torch_dt == torch.float32 else torch.empty(out.shape, dtype=torch_dt, device=dev)
+            po = torch.empty(out.shape, dtype=torch_dt).pin_memory()
+
+            def e2e_step():
+                for i, (bb, g) in enumerate(slices):
+                    st_i = streams[i % len(streams)]
+                    hs, gs = slice(g * G, (g + GPS) * G), slice(g, g + GPS)
+                    with torch.cuda.stream(st_i):
+                        dq[bb:bb + 1, hs].copy_(pq[bb:bb + 1, hs], non_blocking=True)
+                        dk[bb:bb + 1, gs].copy_(pk[bb:bb + 1, gs], non_blocking=True)
+                        dv[bb:bb + 1, gs].copy_(pv[bb:bb + 1, gs], non_blocking=True)
+                        hb.attention_fwd_raw(dq[bb:bb + 1, hs], dk[bb:bb + 1, gs], dv[bb:bb + 1, gs],
+                                             None if s is None else s[gs], None if inv_s is None else inv_s[gs],
+                                             cfg.causal, Bc=cfg.Bc, out_dtype=out_code, out=d_out[bb:bb + 1, hs],
+                                             workspace=ws_s[i % len(streams)], d_status=status)
+                        po[bb:bb + 1, hs].copy_(d_out[bb:bb + 1, hs], non_blocking=True)
+
+            fork()
+            for _ in range(3):
+                e2e_step()
+            join()
+            barrier()
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            n_e2e = max(3, min(args.steps, 10))
+            a.record()
+            fork()
+            for _ in range(n_e2e):
+                e2e_step()
+            join()
+            b.record()
+            barrier()
+            assert int(status.item()) == 0, f"device status {int(status.item())}"
+            # the host copy equals the device-resident result of the timed steps, rounded once to the output dtype
+            assert torch.equal(po.to(dev), out.to(torch_dt)), "end-to-end output differs from the device result"
+            e_ms = max_over_ranks(dist, a.elapsed_time(b), dev)
+            h2d = (pq.numel() + pk.numel() + pv.numel()) * pq.element_size()
+            return {"value": whole_job_tflops(cfg, world, n_e2e, e_ms), "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": po.numel() * po.element_size(),
+                    "ms_per_step": e_ms / n_e2e, "out_dtype": str(torch_dt).replace("torch.", ""),
+                    "how": f"hifa4_attention_fwd_raw per (batch, KV head group) slice, {len(slices)} slices over "
+                           f"{len(streams)} streams, pinned host buffers"}
+
+        e2e_f32 = e2e_run(hb.F32, torch.float32)
+        e2e = e2e_run(hb.F16, torch.float16)
 
     # ---- context (not the product): torch SDPA in BF16 on the same inputs, and, for the headline
     # workload, its N = 8192 sibling (the target sentence names an 8K prefill, the configuration 4K)
@@ -431,28 +526,47 @@ def main():
         except Exception as e:                                         # context only: never fail the bench on it
             context["torch_sdpa_bf16_tflops"] = None
             context["torch_sdpa_error"] = str(e)[:120]
-        if cfg.name == synth.CONFIGS["C2"].name and cfg.N == 4096:
-            c8 = synth.config("C2", N=8192, Bc=cfg.Bc, causal=cfg.causal)
-            q8, k8, v8 = synth.make_qkv_device(c8, dev)
-            qkv8 = hb.alloc_qkv(c8.B, c8.Hq, c8.Hkv, c8.N, c8.d, dt, dev)
-            out8 = torch.empty((c8.B, c8.Hq, c8.N, c8.d), dtype=torch.float32, device=dev)
+        assert int(status.item()) == 0
 
-            def step8():
-                hb.quantize_qkv(q8, k8, v8, s, inv_s, out=qkv8, d_status=status)
-                hb.attention_fwd(qkv8, c8.causal, Bc=c8.Bc, out_dtype=hb.F32, out=out8, d_status=status)
+    # ---- sweep (rank 0, headline run only): every other configuration and the variants, each timed on the
+    # device like the headline (events around each step, L2 flushed between steps), under the same clock record
+    sweep, gemm, sweep_clocks = None, None, None
+    headline = cfg.name == synth.CONFIGS["C2"].name and cfg.N == 4096 and cfg.causal and cfg.Bc == 64 \
+        and not args.qmean and not args.p_f32
+    if rank == 0 and headline and not args.no_sweep:
+        gemm = measure_gemm_peaks(dev)
+        del out
+        sweep = {}
+        sweep_sampler = ClockSampler(local_rank)
+        sweep_sampler.start()
+        sweep_sampler.mark_begin()
 
-            for _ in range(3):
-                flush_l2(); step8()
-            torch.cuda.synchronize()
-            ms8 = 0.0
-            for _ in range(20):
-                flush_l2()
-                a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
-                a.record(); step8(); b.record()
-                torch.cuda.synchronize()
-                ms8 += a.elapsed_time(b)
-            context["C2_at_N8192_step_tflops"] = attn_flops(c8) * 20 / (ms8 * 1e-3) / 1e12
-            del q8, k8, v8, qkv8, out8
+        def cal(c):
+            if not c.smooth_mode:
+                return None, None
+            qc_, kc_ = synth.make_calibration(c, samples=min(c.cal_samples, 4), tokens=min(c.cal_tokens, 256))
+            return hb.smooth_calibrate(qc_.to(dev), kc_.to(dev), c.smooth_mode)
+
+        entries = [("C1", synth.config("C1"), {}),
+                   ("C2@8192 causal (the shape the target sentence names)", synth.config("C2", N=8192), {}),
+                   ("C2 non-causal", synth.config("C2", causal=False), {}),
+                   ("C2 Bc=128", synth.config("C2", Bc=128), {}),
+                   ("C2 Q-Mean", synth.config("C2"), {"qmean": True}),
+                   ("C2 FP32-P variant", synth.config("C2"), {"p_f32": True}),
+                   ("C3", synth.config("C3"), {}), ("C4", synth.config("C4"), {})]
+        for n_ in (1024, 2048, 4096, 8192, 16384, 32768):
+            entries.append((f"C5@{n_} causal", synth.config("C5", N=n_), {}))
+            entries.append((f"C5@{n_} non-causal", synth.config("C5", N=n_, causal=False), {}))
+        for label, c, kw in entries:
+            big_c = c.N >= 16384
+            s_c, is_c = cal(c)
+            r = time_workload(hb, c, dev, steps=3 if big_c else 8, warmup=3, flush_l2=flush_l2, s=s_c, inv_s=is_c, **kw)
+            r["frac_of_measured_bf16_peak"] = r["attention_tflops"] / measured_peaks()["bf16"]
+            sweep[label] = {k_: (round(v_, 5) if isinstance(v_, float) else v_) for k_, v_ in r.items()}
+            torch.cuda.empty_cache()
+        sweep_sampler.mark_end()
+        sweep_clocks = sweep_sampler.stop()
+        sweep_clocks["window"] = "the whole sweep"
         assert int(status.item()) == 0
 
     if rank != 0:
@@ -471,31 +585,41 @@ def main():
         kern = "attention_fwd_ws_kernel<4>"
     else:
         kern = f"attention_fwd_kernel<{cfg.d},{cfg.Bc}>"
+    frac_measured = {"bf16_driver_measured": achieved / peaks["bf16"]}
+    if gemm:
+        if gemm.get("bf16_tflops"):
+            frac_measured["bf16_this_run"] = achieved / gemm["bf16_tflops"]
+            frac_measured["fp4_as_4x_bf16_this_run"] = achieved / (4 * gemm["bf16_tflops"])
+        if gemm.get("fp8_tflops"):
+            frac_measured["fp8_this_run"] = achieved / gemm["fp8_tflops"]
     roofline = {"bound": "tensor", "kernel": kern, "achieved": achieved, "peak": peaks["bf16"],
-                "unit": "TFLOP/s", "frac": achieved / peaks["bf16"],
+                "unit": "TFLOP/s", "frac": achieved / peaks["bf16"], "frac_of_measured": frac_measured,
                 "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, cfg.Bc) if cfg.causal and not args.p_f32 else None),
                 "peak_source": f"{peaks['source']} cuBLAS bf16 burst (the MMA kind issued is kind::f16 on BF16 images)",
                 "avg_launch_ms": attn_avg_ms,
                 "timed_in": "a second pass of the same steps with one event between the two launches "
                             f"({split_step_ms:.4f} ms per step there)",
                 "frac_of_nominal": {k_: achieved / v_ for k_, v_ in NOMINAL.items()}}
-    # The binding resource of the attention kernel is the issue rate of its softmax/quantizer warps, not
-    # the tensor pipe: scores per second against (SMs x 4 schedulers x clock) warp-instructions per second
-    # divided by the warp-instructions the kernel executes per 32 scores (ncu opcode counters, profiles/).
+    # The binding resource of the attention kernel is the instruction issue of its softmax/quantizer warps, not
+    # the tensor pipe.  Roofline on it: scores per second against (SMs x 4 schedulers x clock x 32 lanes) divided
+    # by the issue slots the METHOD needs per score (ALGORITHMIC_SLOTS_PER_SCORE above).  Beside it, as a separate
+    # figure, the issue-slot utilisation: the same rate against the warp instructions the kernel actually executes
+    # per 32 scores (ncu opcode counters, polling loops included).
     n_scores = cfg.B * cfg.Hq * sum(min(cfg.N, ((qb * 128 + 127) // cfg.Bc + 1) * cfg.Bc) if cfg.causal else cfg.N
                                     for qb in range((cfg.N + 127) // 128)) * 128
     sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
     sm_hz = (clocks.get("sm_mhz") or 1965.0) * 1e6
+    ach_scores = n_scores / (attn_avg_ms * 1e-3)
+    peak_scores = sm_count * 4 * sm_hz * 32 / ALGORITHMIC_SLOTS_PER_SCORE
+    roofline_alu = {"bound": "alu", "kernel": kern, "achieved": ach_scores / 1e9, "peak": peak_scores / 1e9,
+                    "unit": "Gscore/s", "frac": ach_scores / peak_scores,
+                    "algorithmic_issue_slots_per_score": ALGORITHMIC_SLOTS_PER_SCORE,
+                    "peak_source": f"{sm_count} SMs x 4 schedulers x {sm_hz / 1e6:.0f} MHz (sampled) x 32 lanes / "
+                                   f"{ALGORITHMIC_SLOTS_PER_SCORE} issue slots per score the method needs"}
     instr_per_warp_score = NCU_INSTR_PER_WARP_SCORE.get(kern)
-    roofline_alu = None
     if instr_per_warp_score:
-        peak_scores = sm_count * 4 * sm_hz * 32 / instr_per_warp_score
-        ach_scores = n_scores / (attn_avg_ms * 1e-3)
-        roofline_alu = {"bound": "alu", "kernel": kern, "achieved": ach_scores / 1e9, "peak": peak_scores / 1e9,
-                        "unit": "Gscore/s", "frac": ach_scores / peak_scores,
-                        "instr_per_warp_score": instr_per_warp_score,
-                        "peak_source": f"{sm_count} SMs x 4 schedulers x {sm_hz / 1e6:.0f} MHz (sampled) x 32 lanes / "
-                                       "executed warp instructions per warp-score (ncu)"}
+        roofline_alu["issue_slot_utilisation"] = ach_scores * instr_per_warp_score / (sm_count * 4 * sm_hz * 32)
+        roofline_alu["executed_instr_per_warp_score"] = instr_per_warp_score
     q_bytes = sum(t.numel() for t in (q, k, v)) * (2 + 0.5625)
     quant = {"avg_ms": sum(quant_ms) / len(quant_ms), "algorithmic_gbs": q_bytes / (sum(quant_ms) / len(quant_ms) * 1e-3) / 1e9,
              "hbm_peak_gbs": peaks["hbm"]}
@@ -525,8 +649,9 @@ def main():
                        "l2": "flushed between steps (256 MiB write, then a 256 MiB read that drains the dirty lines), outside the per-step events",
                        "parallelism": f"replicated batches x{world}"},
             "frac_of_nominal_peak": {k_: value / world / v_ for k_, v_ in NOMINAL.items()},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-            "roofline_alu": roofline_alu, "quantize": quant, "cpu_baseline": cpu, "context": context}
+            "clocks": clocks, "e2e": e2e, "e2e_f32_out": e2e_f32, "gpu_launches": launches, "roofline": roofline,
+            "roofline_alu": roofline_alu, "quantize": quant, "cpu_baseline": cpu, "context": context,
+            "measured_gemm_peaks_this_run": gemm, "sweep": sweep, "sweep_clocks": sweep_clocks}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()

@@ -46,6 +46,7 @@ typedef enum { HIFA4_F16 = 0, HIFA4_BF16 = 1, HIFA4_F32 = 2 } hifa4_dtype;
 enum { HIFA4_Q = 0, HIFA4_K = 1, HIFA4_V = 2 };               /* `which` */
 enum { HIFA4_PART_CODES = 0, HIFA4_PART_META = 1, HIFA4_PART_MMA = 2, HIFA4_PART_AUX = 3 }; /* `part` */
 enum { HIFA4_MAX_HEADS = 256, HIFA4_MAX_DEBUG_BLOCKS = 16 };
+enum { HIFA4_AGG_RMS = 0, HIFA4_AGG_MEAN = 0x100, HIFA4_AGG_P99 = 0x200 };   /* OR-ed into calibration `mode` */
 #define HIFA4_STATIC_CALIB_MAX_FLOATS (1u << 20)   /* scratch limit of hifa4_smooth_calibrate_static */
 
 /* Problem shape.  Q is [B,Hq,N,d]; K and V are [B,Hkv,N,d] ("GQA and batch
@@ -153,6 +154,18 @@ typedef struct {
 
 const char* hifa4_status_string(int status);
 
+/* Self-test of the failure path of the device-side waits (no counterpart in the paper; for deployment
+ * checks and for the test-suite).  Launches the Bc = 64, d = 128 attention kernel in an instantiation
+ * whose softmax warps withhold the arrival that releases the P V product and whose issuer gives up
+ * waiting for it after 2^12 polls (a fraction of a millisecond) instead of 2^20.  When that wait runs out
+ * every TMA load has landed and no MMA is in flight; the kernel records HIFA4_ERR_TIMEOUT + 16 * 7 (site 7:
+ * the issuer's wait for P V) in *d_status (required, device int, zero on entry), raises the CTA's abort flag,
+ * every role leaves through the common exit that frees tensor memory, and the call returns normally.
+ * `out` is not written.  Arguments as hifa4_attention_fwd (prm: Bc = 64, no variant flags; shape: d = 128);
+ * a one-CTA problem (N <= 128, one head) is what the test-suite uses.  Nothing hangs, faults or traps. */
+int hifa4_selftest_wait_timeout(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
+                                void* out, int* d_status, void* stream);
+
 /* Calls made so far in this process: out[0] calibrate, out[1] quantize,
  * out[2] attention, out[3] kernels launched (all entry points). */
 void hifa4_get_counters(unsigned long long out[4]);
@@ -166,7 +179,10 @@ void hifa4_get_counters(unsigned long long out[4]);
  *   aggregate is zero.  mode: 0 bypass (s = 1), 1 strong (alpha 0.5), 2 mild
  *   (alpha 0.25), 4 caller's alpha; 3 (gate decides) returns
  *   HIFA4_ERR_UNSUPPORTED here: use hifa4_smooth_calibrate_auto, which takes
- *   the extra scratch the gate statistics need.
+ *   the extra scratch the gate statistics need.  OR-ing HIFA4_AGG_MEAN or
+ *   HIFA4_AGG_P99 into mode replaces the root-mean-square over samples by the
+ *   mean or by the nearest-rank 99th percentile of the per-sample maxima (the
+ *   two alternatives of the paper's aggregator comparison, table "calib").
  *   Outputs (device): s, inv_s [Hkv,d] floats, inv_s = fl32(1/s).
  *   absmax_ws: device scratch of 2*S*Hkv*d floats; the call clears it.
  *   host_stats: optional HOST struct, filled without synchronizing. */

@@ -17,6 +17,7 @@ F16, BF16, F32 = 0, 1, 2
 Q, K, V = 0, 1, 2
 CODES, META, MMA, AUX = 0, 1, 2, 3
 MODE_BYPASS, MODE_STRONG, MODE_MILD, MODE_AUTO, MODE_CUSTOM = 0, 1, 2, 3, 4
+AGG_RMS, AGG_MEAN, AGG_P99 = 0, 0x100, 0x200            # OR-ed into the calibration mode
 MAX_DEBUG_BLOCKS = 16
 
 _DT = {torch.float16: F16, torch.bfloat16: BF16, torch.float32: F32}
@@ -103,6 +104,9 @@ def lib():
         L.hifa4_attention_fwd.restype = C.c_int
         L.hifa4_attention_fwd.argtypes = [C.POINTER(_Shape), C.POINTER(_QKV), C.POINTER(_AttnParams),
                                           C.c_void_p, C.c_void_p, C.POINTER(_Debug), C.c_void_p, C.c_void_p]
+        L.hifa4_selftest_wait_timeout.restype = C.c_int
+        L.hifa4_selftest_wait_timeout.argtypes = [C.POINTER(_Shape), C.POINTER(_QKV), C.POINTER(_AttnParams),
+                                                  C.c_void_p, C.c_void_p, C.c_void_p]
         L.hifa4_attention_fwd_stats.restype = C.c_int
         L.hifa4_attention_fwd_stats.argtypes = [C.POINTER(_Shape), C.POINTER(_QKV), C.POINTER(_AttnParams),
                                                 C.c_void_p, C.c_void_p, C.POINTER(_MassStats), C.c_void_p,
@@ -120,7 +124,8 @@ STATIC_CALIB_MAX_FLOATS = 1 << 20
 EXPORTS = ("hifa4_status_string", "hifa4_get_counters", "hifa4_smooth_calibrate",
            "hifa4_smooth_calibrate_static", "hifa4_smooth_calibrate_auto", "hifa4_quant_bytes",
            "hifa4_quantize_qkv", "hifa4_attention_workspace_bytes", "hifa4_attention_fwd",
-           "hifa4_attention_fwd_stats", "hifa4_attention_raw_workspace_bytes", "hifa4_attention_fwd_raw")
+           "hifa4_attention_fwd_stats", "hifa4_attention_raw_workspace_bytes", "hifa4_attention_fwd_raw",
+           "hifa4_selftest_wait_timeout")
 
 
 def status_string(status: int) -> str:
@@ -220,8 +225,9 @@ def alloc_qkv(B, Hq, Hkv, N, d, in_dtype, device, q_to_kv=None, qmean=False) -> 
     return QuantizedQKV(B, Hq, Hkv, N, d, in_dtype, q_to_kv, **bufs)
 
 
-def smooth_calibrate(q_cal, k_cal, mode, alpha=0.0, q_to_kv=None):
-    """q_cal [S,Hq,Ncal,d], k_cal [S,Hkv,Ncal,d] device tensors -> (s, inv_s) [Hkv,d] float32."""
+def smooth_calibrate(q_cal, k_cal, mode, alpha=0.0, q_to_kv=None, aggregator=AGG_RMS):
+    """q_cal [S,Hq,Ncal,d], k_cal [S,Hkv,Ncal,d] device tensors -> (s, inv_s) [Hkv,d] float32.
+    aggregator: AGG_RMS (the paper's choice), AGG_MEAN or AGG_P99 over the calibration samples."""
     assert q_cal.is_cuda and k_cal.is_cuda and q_cal.is_contiguous() and k_cal.is_contiguous()
     S, Hq, Ncal, d = q_cal.shape
     Hkv = k_cal.shape[1]
@@ -232,7 +238,7 @@ def smooth_calibrate(q_cal, k_cal, mode, alpha=0.0, q_to_kv=None):
     keep, mp = _map_arr(q_to_kv)
     stats = _CalibStats()
     rc = lib().hifa4_smooth_calibrate(_ptr(q_cal), _ptr(k_cal), S, Hq, Hkv, Ncal, d, mp, _DT[q_cal.dtype],
-                                      int(mode), float(alpha), _ptr(s), _ptr(inv_s), _ptr(ws),
+                                      int(mode) | int(aggregator), float(alpha), _ptr(s), _ptr(inv_s), _ptr(ws),
                                       C.byref(stats), _stream())
     _check(rc, "hifa4_smooth_calibrate")
     return s, inv_s
@@ -328,6 +334,19 @@ def attention_fwd(qkv: QuantizedQKV, causal: bool, Bc: int = 64, out_dtype=F32, 
                                    _ptr(d_status), _stream())
     _check(rc, "hifa4_attention_fwd")
     return (out, dump) if debug_blocks else out
+
+
+def selftest_wait_timeout(qkv: QuantizedQKV, causal: bool, d_status, out=None):
+    """Launches the self-test instantiation whose wait for P V runs out (see include/hifa4.h).  d_status: device
+    int32 tensor (zero on entry); afterwards it holds HIFA4_ERR_TIMEOUT + 16 * 7.  Returns the (unwritten) out."""
+    sh = _shape(qkv.B, qkv.Hq, qkv.Hkv, qkv.N, qkv.d, qkv.in_dtype, qkv.q_to_kv)
+    prm = _params(causal, 64, F32)
+    if out is None:
+        out = torch.empty((qkv.B, qkv.Hq, qkv.N, qkv.d), dtype=torch.float32, device=qkv.q_mma.device)
+    st = qkv.struct()
+    rc = lib().hifa4_selftest_wait_timeout(C.byref(sh), C.byref(st), C.byref(prm), _ptr(out), _ptr(d_status), _stream())
+    _check(rc, "hifa4_selftest_wait_timeout")
+    return out
 
 
 def attention_fwd_stats(qkv: QuantizedQKV, causal: bool, n_bins: int, lo: float, hi: float, Bc: int = 64,

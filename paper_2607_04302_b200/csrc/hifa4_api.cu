@@ -85,6 +85,10 @@ int hifa4_smooth_calibrate(const void* q_cal, const void* k_cal, int S, int Hq, 
     if (S <= 0 || Ncal <= 0) return HIFA4_ERR_INVALID_ARG;
     if (dt != HIFA4_F16 && dt != HIFA4_BF16) return HIFA4_ERR_INVALID_ARG;
     if (d != 64 && d != 128 && d != 256) return HIFA4_ERR_UNSUPPORTED;
+    if (mode < 0 || (mode & ~0x3FF)) return HIFA4_ERR_INVALID_ARG;
+    const int aggregator = mode >> 8;                              // HIFA4_AGG_* flag
+    mode &= 0xFF;
+    if (aggregator > 2) return HIFA4_ERR_INVALID_ARG;
     if (mode == 3) return HIFA4_ERR_UNSUPPORTED;
     if (mode < 0 || mode > 4) return HIFA4_ERR_INVALID_ARG;
     if (mode == 4 && !(alpha >= 0.f && alpha <= 1.f)) return HIFA4_ERR_INVALID_ARG;
@@ -102,7 +106,7 @@ int hifa4_smooth_calibrate(const void* q_cal, const void* k_cal, int S, int Hq, 
         if (launch_absmax(dt, k_cal, kmap, S, Hkv, Hkv, Ncal, d, kmax, st) != cudaSuccess) return HIFA4_ERR_CUDA;
         if (launch_absmax(dt, q_cal, qmap, S, Hq, Hkv, Ncal, d, qmax, st) != cudaSuccess) return HIFA4_ERR_CUDA;
     }
-    if (launch_smooth_finalize(kmax, qmax, S, Hkv * d, a, mode == 0, nullptr, s, inv_s, st) != cudaSuccess)
+    if (launch_smooth_finalize(kmax, qmax, S, Hkv * d, a, mode == 0, aggregator, nullptr, s, inv_s, st) != cudaSuccess)
         return HIFA4_ERR_CUDA;
     if (host_stats) {
         host_stats->rho_K = NAN;
@@ -137,7 +141,7 @@ int hifa4_smooth_calibrate_auto(const void* q_cal, const void* k_cal, int S, int
     if (launch_absmax(dt, k_cal, kmap, S, Hkv, Hkv, Ncal, d, kmax, st) != cudaSuccess) return HIFA4_ERR_CUDA;
     if (launch_absmax(dt, q_cal, qmap, S, Hq, Hkv, Ncal, d, qmax, st) != cudaSuccess) return HIFA4_ERR_CUDA;
     if (launch_gate(dt, k_cal, nk, kmax, qmax, (int)n, gate_ws, d_stats, st) != cudaSuccess) return HIFA4_ERR_CUDA;
-    if (launch_smooth_finalize(kmax, qmax, S, Hkv * d, 0.0, 0, gate_result(gate_ws), s, inv_s, st) != cudaSuccess)
+    if (launch_smooth_finalize(kmax, qmax, S, Hkv * d, 0.0, 0, 0, gate_result(gate_ws), s, inv_s, st) != cudaSuccess)
         return HIFA4_ERR_CUDA;
     return HIFA4_OK;
 }
@@ -203,7 +207,7 @@ size_t hifa4_attention_workspace_bytes(const hifa4_shape* shape, const hifa4_att
 
 static int attention_common(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
                             void* out, const hifa4_debug* dbg, const hifa4_mass_stats* stats, int* d_status,
-                            void* stream)
+                            void* stream, bool selftest = false)
 {
     g_calls[2].fetch_add(1, std::memory_order_relaxed);
     int rc = check_attn(shape, prm);
@@ -223,7 +227,7 @@ static int attention_common(const hifa4_shape* shape, const hifa4_qkv* qkv, cons
     HeadMap qmap, kmap;
     if ((rc = build_map(shape->Hq, shape->Hkv, shape->q_to_kv, qmap, kmap))) return rc;
     if ((rc = check_arch())) return rc;
-    return launch_attention(*shape, qmap, *qkv, *prm, out, dbg, stats, d_status, (cudaStream_t)stream);
+    return launch_attention(*shape, qmap, *qkv, *prm, out, dbg, stats, d_status, (cudaStream_t)stream, selftest);
 }
 
 int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
@@ -232,6 +236,13 @@ int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv, const hi
 {
     (void)workspace;
     return attention_common(shape, qkv, prm, out, dbg, nullptr, d_status, stream);
+}
+
+int hifa4_selftest_wait_timeout(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
+                                void* out, int* d_status, void* stream)
+{
+    if (!d_status) return HIFA4_ERR_INVALID_ARG;
+    return attention_common(shape, qkv, prm, out, nullptr, nullptr, d_status, stream, true);
 }
 
 int hifa4_attention_fwd_stats(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,

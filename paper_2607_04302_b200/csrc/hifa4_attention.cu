@@ -344,7 +344,7 @@ static int launch_cfg(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArg
 
 int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv& qkv,
                      const hifa4_attn_params& prm, void* out, const hifa4_debug* dbg,
-                     const hifa4_mass_stats* stats, int* d_status, cudaStream_t st)
+                     const hifa4_mass_stats* stats, int* d_status, cudaStream_t st, bool selftest)
 {
     AttnArgs a;
     memset(&a, 0, sizeof(a));
@@ -371,6 +371,10 @@ int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv&
     a.head_major = (double)sh.B * sh.Hkv * sh.N * sh.d * 4.0 > 200e6 ? 1 : 0;
     a.normalizer = prm.normalizer ? 1 : 0;
     a.p_f32 = prm.p_dtype == HIFA4_F32 ? 1 : 0;
+    if (selftest) {                               // the instantiation whose wait for P V runs out
+        if (a.p_f32 || a.normalizer || a.qmean || stats || dbg || prm.Bc != 64 || sh.d != 128) return HIFA4_ERR_UNSUPPORTED;
+        return launch_attention_ws64_selftest(sh, qkv, a, st);
+    }
     if (a.p_f32) {                                // variant built for the 64-key warp-specialised kernels only
         if (a.normalizer || stats || prm.Bc != 64 || (sh.d != 128 && sh.d != 256)) return HIFA4_ERR_UNSUPPORTED;
         return launch_attention_ws64(sh, qkv, a, st);

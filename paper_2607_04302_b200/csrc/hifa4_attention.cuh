@@ -294,5 +294,7 @@ int launch_attention_ws(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnA
 
 // Warp-specialised kernels for Bc = 64, d = 64, 128 or 256 (hifa4_attention_ws64.cu).
 int launch_attention_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st);
+// Self-test instantiation (d = 128): one bounded wait is made to run out (see hifa4_selftest_wait_timeout).
+int launch_attention_ws64_selftest(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st);
 
 }  // namespace hifa4

@@ -79,10 +79,11 @@ constexpr uint32_t WAIT_POLLS = 1u << 20;
 
 // Bounded wait with non-blocking polls (softmax warps and issuers: a late wake-up sits on the critical path,
 // and a thread suspended in try_wait was seen to notice a completed phase about 1000 clk late).
-static __device__ __forceinline__ bool wait64(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+static __device__ __forceinline__ bool wait64(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                              uint32_t polls = ws64::WAIT_POLLS)
 {
 #pragma unroll 1
-    for (uint32_t i = 0; i < ws64::WAIT_POLLS; ++i) {
+    for (uint32_t i = 0; i < polls; ++i) {
         if (mbar_test_wait(bar, parity)) return true;
         if ((i & 63u) == 63u && *abort_flag) return false;
     }
@@ -108,7 +109,10 @@ static __device__ __forceinline__ void arrive_lane0(uint32_t bar, int lane)
                  ::"r"(bar), "r"(lane) : "memory");
 }
 
-template <int DH, bool DBG, bool PF32, bool QM>
+// SELFTEST: the instantiation behind hifa4_selftest_wait_timeout.  Its softmax warps withhold the arrival that
+// releases P V and the issuer's wait for it gives up after 2^12 polls instead of 2^20; by then every TMA load
+// has landed and no MMA is in flight, so the CTA leaves through the ordinary failure exit.
+template <int DH, bool DBG, bool PF32, bool QM, bool SELFTEST = false>
 __global__ void __launch_bounds__(WS64<DH>::THREADS, WS64<DH>::CTAS_PER_SM)
 attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                            const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnArgs args)
@@ -254,7 +258,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             for (int jt = 0; jt < n_tiles; ++jt) {            // V^T tile landed, P-hat(jt) stored, history rescaled
                 const int st = jt & 1;
                 const uint32_t ph = (uint32_t)(jt >> 1) & 1u;
-                if (!wait64(bar(BAR_PVGO + st), ph, abort_flag)) { fail(7); break; }
+                if (!wait64(bar(BAR_PVGO + st), ph, abort_flag, SELFTEST ? (1u << 12) : WAIT_POLLS)) { fail(7); break; }
                 tc_fence_after();
                 const uint32_t b0 = v_lo + st * (V_STAGE >> 4);
                 const uint32_t acc0 = jt > 0 ? 1u : 0u;
@@ -438,7 +442,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
-            arrive_lane0(bar(BAR_PVGO + st), lane);
+            if (!SELFTEST) arrive_lane0(bar(BAR_PVGO + st), lane);
         }
 
         // finalize: out = O / l with l rounded to FP16 (line 13); half kq writes channels (d/2)*kq..
@@ -521,7 +525,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     if (warp == W_QK) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
 }
 
-template <int DH, bool DBG, bool PF32, bool QM>
+template <int DH, bool DBG, bool PF32, bool QM, bool SELFTEST = false>
 static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
     using C = WS64<DH>;
@@ -529,7 +533,7 @@ static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnAr
     if (!make_bf16_map(&mq, qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, DH, 128)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, DH, C::BC)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, DH, sh.N, DH)) return HIFA4_ERR_CUDA;
-    auto kern = attention_fwd_ws64_kernel<DH, DBG, PF32, QM>;
+    auto kern = attention_fwd_ws64_kernel<DH, DBG, PF32, QM, SELFTEST>;
     static SmemOptIn opt_in;
     if (!opt_in.ensure(kern, C::SMEM_BYTES)) return HIFA4_ERR_CUDA;
     dim3 grid((unsigned)(((sh.N + 127) / 128) * sh.Hq * sh.B));
@@ -562,6 +566,12 @@ static int launch_ws64_d(const hifa4_shape& sh, const hifa4_qkv& qkv, const Attn
     if (args.qmean)
         return dbg ? launch_ws64<DH, true, false, true>(sh, qkv, args, st) : launch_ws64<DH, false, false, true>(sh, qkv, args, st);
     return dbg ? launch_ws64<DH, true, false, false>(sh, qkv, args, st) : launch_ws64<DH, false, false, false>(sh, qkv, args, st);
+}
+
+int launch_attention_ws64_selftest(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
+{
+    if (sh.d != 128) return HIFA4_ERR_UNSUPPORTED;
+    return launch_ws64<128, false, false, false, true>(sh, qkv, args, st);
 }
 
 int launch_attention_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)

@@ -39,8 +39,10 @@ cudaError_t launch_quantize_qkv(int dtype, const hifa4_shape& sh, const HeadMap&
 cudaError_t launch_absmax(int dtype, const void* x, const HeadMap& map, int S, int H, int Hkv,
                           int Ncal, int d, float* ws, cudaStream_t st);
 // gate: null, or the device {alpha, bypass} pair written by launch_gate (overrides alpha / bypass).
+// aggregator: 0 root-mean-square, 1 mean, 2 nearest-rank 99th percentile of the per-sample maxima.
 cudaError_t launch_smooth_finalize(const float* kmax, const float* qmax, int S, int n, double alpha,
-                                   int bypass, const double* gate, float* s, float* inv_s, cudaStream_t st);
+                                   int bypass, int aggregator, const double* gate, float* s, float* inv_s,
+                                   cudaStream_t st);
 // Gate statistics and decision on the device.  gate_ws: HIFA4_GATE_WS_BYTES bytes; d_stats: 4 floats or null.
 cudaError_t launch_gate(int dtype, const void* k_cal, long long nk, const float* kmax, const float* qmax,
                         int n_max, void* gate_ws, float* d_stats, cudaStream_t st);
@@ -49,6 +51,6 @@ const double* gate_result(void* gate_ws);
 // Attention forward on the BF16 operand images; returns a hifa4_status.
 int launch_attention(const hifa4_shape& shape, const HeadMap& map, const hifa4_qkv& qkv,
                      const hifa4_attn_params& prm, void* out, const hifa4_debug* dbg,
-                     const hifa4_mass_stats* stats, int* d_status, cudaStream_t st);
+                     const hifa4_mass_stats* stats, int* d_status, cudaStream_t st, bool selftest = false);
 
 }  // namespace hifa4

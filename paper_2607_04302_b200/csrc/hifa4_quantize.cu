@@ -293,22 +293,41 @@ absmax_kernel(const uint16_t* __restrict__ x, HeadMap map, int H, int Hkv, int N
     }
 }
 
-// s = Kagg^alpha / Qagg^(1-alpha) with RMS aggregation over samples; 1 where degenerate.
+// s = Kagg^alpha / Qagg^(1-alpha); 1 where degenerate.  The per-sample maxima are combined over the S samples
+// by root-mean-square (aggregator 0, the paper's choice), mean (1) or nearest-rank 99th percentile (2).
 // gate (optional, device): {alpha, bypass flag} chosen by the applicability gate; overrides the arguments.
+__device__ __forceinline__ double percentile99(const float* __restrict__ v, int S, long long stride)
+{
+    const long long rank = (long long)ceil(0.99 * (double)S) < 1 ? 1 : (long long)ceil(0.99 * (double)S);
+    for (int a = 0; a < S; ++a) {                            // selection by counting: S is small
+        const float va = v[a * stride];
+        long long below = 0, not_above = 0;
+        for (int b = 0; b < S; ++b) { const float vb = v[b * stride]; below += vb < va; not_above += vb <= va; }
+        if (below < rank && rank <= not_above) return (double)va;
+    }
+    return 0.0;
+}
 __global__ void smooth_finalize_kernel(const float* __restrict__ kmax, const float* __restrict__ qmax,
-                                       int S, int n, double alpha, int bypass, const double* __restrict__ gate,
-                                       float* __restrict__ s, float* __restrict__ inv_s)
+                                       int S, int n, double alpha, int bypass, int aggregator,
+                                       const double* __restrict__ gate, float* __restrict__ s, float* __restrict__ inv_s)
 {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     if (gate) { alpha = gate[0]; bypass = gate[1] != 0.0; }
-    double ks = 0, qs = 0;
-    for (int m = 0; m < S; ++m) {
-        double a = kmax[(long long)m * n + i], b = qmax[(long long)m * n + i];
-        ks += a * a;
-        qs += b * b;
+    double kagg, qagg;
+    if (aggregator == 2) {
+        kagg = percentile99(kmax + i, S, n);
+        qagg = percentile99(qmax + i, S, n);
+    } else {
+        double ks = 0, qs = 0;
+        for (int m = 0; m < S; ++m) {
+            double a = kmax[(long long)m * n + i], b = qmax[(long long)m * n + i];
+            ks += aggregator == 1 ? a : a * a;
+            qs += aggregator == 1 ? b : b * b;
+        }
+        kagg = aggregator == 1 ? ks / S : sqrt(ks / S);
+        qagg = aggregator == 1 ? qs / S : sqrt(qs / S);
     }
-    double kagg = sqrt(ks / S), qagg = sqrt(qs / S);
     double sv = 1.0;
     if (!bypass && kagg > 0 && qagg > 0) sv = pow(kagg, alpha) / pow(qagg, 1.0 - alpha);
     float sf = (float)sv;
@@ -364,9 +383,10 @@ cudaError_t launch_absmax(int dtype, const void* x, const HeadMap& map, int S, i
 }
 
 cudaError_t launch_smooth_finalize(const float* kmax, const float* qmax, int S, int n, double alpha,
-                                   int bypass, const double* gate, float* s, float* inv_s, cudaStream_t st)
+                                   int bypass, int aggregator, const double* gate, float* s, float* inv_s,
+                                   cudaStream_t st)
 {
-    smooth_finalize_kernel<<<(n + 127) / 128, 128, 0, st>>>(kmax, qmax, S, n, alpha, bypass, gate, s, inv_s);
+    smooth_finalize_kernel<<<(n + 127) / 128, 128, 0, st>>>(kmax, qmax, S, n, alpha, bypass, aggregator, gate, s, inv_s);
     count_launch();
     return cudaGetLastError();
 }

@@ -278,3 +278,30 @@ def test_nonzero_status_word_makes_every_kernel_family_a_no_op(hb, par, d, Bc, n
     hb.attention_fwd(qkv, True, Bc=Bc, out=out, d_status=status, normalizer=normalizer)
     torch.cuda.synchronize()
     assert int(status.item()) == 0 and torch.equal(out, good) and torch.isfinite(out).all()
+
+
+def test_expired_device_wait_is_reported_and_leaves_the_device_usable(hb, par):
+    """The failure path of the bounded device-side waits, exercised without hanging or faulting anything: the
+    self-test instantiation withholds the arrival that releases P V, the issuer's wait runs out after 2^12 polls,
+    the status word reads HIFA4_ERR_TIMEOUT + 16 * site (site 7 = that wait), the call returns, the output buffer
+    is untouched, and the next ordinary call on the same buffers passes parity (tensor memory was freed, no
+    barrier stayed armed)."""
+    cfg = synth.config("C3", N=128, Hq=1, Hkv=1, causal=False)           # one CTA, two key tiles
+    q, k, v = (t.to(DEV) for t in synth.make_qkv(cfg))
+    qkv = hb.quantize_qkv(q, k, v)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = torch.full((1, 1, cfg.N, cfg.d), 3.0, dtype=torch.float32, device=DEV)
+    hb.selftest_wait_timeout(qkv, False, status, out=out)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 6 + 16 * 7
+    assert hb.status_string(6).lower().find("wait") >= 0 or hb.status_string(6)
+    assert bool((out == 3.0).all())
+    # a call that finds the status word set does nothing either; after clearing it everything works again
+    hb.attention_fwd(qkv, False, Bc=64, out=out, d_status=status)
+    torch.cuda.synchronize()
+    assert bool((out == 3.0).all()) and int(status.item()) == 6 + 16 * 7
+    res = par.run_case(cfg, DEV)
+    print(par.assert_within_bars(res, "after the expired wait"))
+    with pytest.raises(hb.Hifa4Error):                                  # the self-test refuses shapes it was not built for
+        hb.selftest_wait_timeout(hb.quantize_qkv(*(t.to(DEV) for t in synth.make_qkv(synth.config("C3", N=128, Hq=1, Hkv=1, d=64)))),
+                                 False, status)

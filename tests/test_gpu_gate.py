@@ -76,3 +76,25 @@ def test_gate_percentile_is_exact_on_ties_and_edges(hb, oracle):
     k3 = flat.reshape(1, 1, 64, 64).to(torch.bfloat16)
     _, _, st3 = hb.smooth_calibrate_auto(q.to(DEV), k3.to(DEV))
     assert st3.cpu().tolist() == [1.0, 64.0, 0.0, 0.0]
+
+
+@pytest.mark.parametrize("agg", ["rms", "mean", "p99"])
+def test_calibration_aggregators_match_the_oracle(hb, oracle, agg):
+    """Mean and 99th-percentile aggregation of the per-sample channel maxima (the alternatives of the paper's
+    aggregator comparison) beside the adopted root-mean-square: factors equal to the oracle's to 1e-6."""
+    gen = torch.Generator().manual_seed(31)
+    S, Hq, Hkv, Ncal, d = 120, 4, 2, 8, 128
+    spread = torch.exp(torch.randn((S, 1, 1, 1), generator=gen) * 0.4)
+    q = (torch.randn((S, Hq, Ncal, d), generator=gen) * spread).to(torch.bfloat16)
+    k = (torch.randn((S, Hkv, Ncal, d), generator=gen) * spread * 3).to(torch.bfloat16)
+    flag_o = {"rms": oracle.AGG_RMS, "mean": oracle.AGG_MEAN, "p99": oracle.AGG_P99}[agg]
+    flag_g = {"rms": hb.AGG_RMS, "mean": hb.AGG_MEAN, "p99": hb.AGG_P99}[agg]
+    ref = oracle.smooth_calibrate(q.float().numpy(), k.float().numpy(), 1, aggregator=flag_o)
+    s, inv_s = hb.smooth_calibrate(q.to(DEV), k.to(DEV), 1, aggregator=flag_g)
+    assert np.allclose(s.cpu().numpy(), ref["s"], rtol=1e-6)
+    assert torch.equal(inv_s, 1.0 / s)
+    if agg != "rms":
+        base, _ = hb.smooth_calibrate(q.to(DEV), k.to(DEV), 1)
+        assert not torch.equal(base, s)
+    with pytest.raises(hb.Hifa4Error):
+        hb.smooth_calibrate(q.to(DEV), k.to(DEV), 1, aggregator=0x300)
