@@ -34,7 +34,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-Xlinker", "-rpath,/usr/local/cuda/lib64"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("HIFA4_NVCC_FLAGS", "").split()       # extra compiler flags (experiments)
     cmd += sources() + ["-o", tmp]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

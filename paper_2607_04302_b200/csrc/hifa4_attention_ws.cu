@@ -44,18 +44,16 @@ enum { BAR_QFULL = 0, BAR_QFREE = 2, BAR_KF = 4, BAR_KE = 6, BAR_VF = 8, BAR_VE 
 constexpr uint32_t WAIT_POLLS = 1u << 20;           // each poll blocks for a hardware-defined slice
 }  // namespace ws
 
-// Bounded waits.  wait_or_abort polls back to back (softmax warps: their waits are usually already
-// satisfied, and a late wake-up would sit on the critical path).  wait_sleepy lets the hardware
-// suspend the thread for up to a few microseconds per poll (it wakes when the phase completes), so
-// the producer and issuer warps, which wait most of the time, do not burn the issue slots and the
-// memory-I/O queue that the softmax warps need.
+// Bounded waits.  wait_or_abort polls without blocking (softmax warps and the issuer: a late wake-up sits on
+// the critical path, and a thread suspended in try_wait was seen to notice a completed phase about 1000 clk
+// late).  wait_sleepy lets the hardware suspend the thread for up to a few microseconds per poll, for the
+// producer warp, which waits most of the time and has slack.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag)
 {
-    for (uint32_t i = 0; i < ws::WAIT_POLLS / 64; ++i) {
 #pragma unroll 1
-        for (int j = 0; j < 64; ++j)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
+    for (uint32_t i = 0; i < ws::WAIT_POLLS; ++i) {
+        if (mbar_test_wait(bar, parity)) return true;
+        if ((i & 63u) == 63u && *abort_flag) return false;
     }
     return false;
 }

@@ -44,34 +44,6 @@ __device__ __forceinline__ float e6m2_inv4(int code)        // 4 / S
     return __uint_as_float(r + ((uint32_t)(50 - (code >> 2)) << 23));
 }
 
-// Shift needed by a 4-element subgroup with maximum At: 0, 1 or 2.
-__device__ __forceinline__ int hif4_need(float At, float S)
-{
-    return (At > 1.75f * S) + (At > 3.5f * S);
-}
-
-// Level-2 bit of a pair of subgroups and their level-3 bits.
-// a = 1 iff max(need) = 2 or min(need) >= 1  <=>  need0 + need1 >= 2.
-__device__ __forceinline__ void hif4_pair_bits(int n0, int n1, int& a, int& b0, int& b1)
-{
-    a = (n0 + n1) >= 2;
-    b0 = min(max(n0 - a, 0), 1);
-    b1 = min(max(n1 - a, 0), 1);
-}
-
-__device__ __forceinline__ float scale_pow2(float x, int k)  // x * 2^k, x normal, no overflow
-{
-    return __uint_as_float(__float_as_uint(x) + ((uint32_t)k << 23));
-}
-
-// Element code: nearest multiple of step (ties to even), saturating at 7.
-__device__ __forceinline__ int hif4_code(float ax, float inv_step)
-{
-    float q = __fmul_rz(ax, inv_step);
-    int m = __float2int_rn(q);
-    return min(m, 7);
-}
-
 template <typename T> struct In16;
 template <> struct In16<__half> {
     static __device__ __forceinline__ float to_f(uint16_t u) { return __half2float(__ushort_as_half(u)); }

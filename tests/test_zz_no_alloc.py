@@ -25,10 +25,17 @@ def test_static_scratch_entry_point_matches_workspace_entry_point():
         qc, kc = qc.to(DEV), kc.to(DEV)
         s = torch.full((cfg.Hkv, cfg.d), -1.0, dtype=torch.float32, device=DEV)
         inv_s = torch.full_like(s, -1.0)
+        torch.cuda.synchronize()
         before = torch.cuda.memory_allocated(DEV)
+        free_before = torch.cuda.mem_get_info(DEV)[0]
         hb.smooth_calibrate_static(qc, kc, cfg.smooth_mode, s=s, inv_s=inv_s)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated(DEV) == before          # torch saw no allocation either
+        assert torch.cuda.memory_allocated(DEV) == before          # torch saw no allocation
+        # and neither did the driver: by the third call every kernel of the entry point is loaded, so the
+        # device's free memory cannot move unless the library itself allocated (cudaMalloc, a stream-ordered
+        # allocation) -- which torch's own counter above would not see
+        if call == 2:
+            assert torch.cuda.mem_get_info(DEV)[0] == free_before
         s_ref, inv_ref = hb.smooth_calibrate(qc, kc, cfg.smooth_mode)
         torch.cuda.synchronize()
         # same kernels on the same data: identical bits, which is inside the 1e-6 relative tolerance
