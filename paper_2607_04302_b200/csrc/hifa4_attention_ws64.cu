@@ -89,17 +89,6 @@ static __device__ __forceinline__ bool wait64(uint32_t bar, uint32_t parity, vol
     }
     return false;
 }
-// Bounded wait of the producer warp, which waits most of the time and has slack: the hardware may keep the
-// thread suspended for a few microseconds per poll (it wakes when the phase completes).
-static __device__ __forceinline__ bool wait_idle(uint32_t bar, uint32_t parity, volatile int* abort_flag)
-{
-#pragma unroll 1
-    for (uint32_t i = 0; i < ws64::WAIT_POLLS / 4; ++i) {
-        if (mbar_try_wait_hint(bar, parity, 4000u)) return true;
-        if (*abort_flag) return false;
-    }
-    return false;
-}
 // One arrival from lane 0 of a converged warp, without a branch.
 static __device__ __forceinline__ void arrive_lane0(uint32_t bar, int lane)
 {
@@ -242,7 +231,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 umma_commit(bar(BAR_SF + st));
                 umma_commit(bar(BAR_KE + st));
                 if (jt + 2 < n_tiles) {                        // refill the stage once this MMA has read it
-                    if (!wait_idle(bar(BAR_KE + st), ph, abort_flag)) { fail(1); break; }
+                    if (!wait64(bar(BAR_KE + st), ph, abort_flag)) { fail(1); break; }
                     load_k(jt + 2);
                 }
             }
@@ -271,7 +260,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 umma_commit(bar(BAR_PV + st));
                 umma_commit(bar(BAR_VE + st));
                 if (jt + 2 < n_tiles) {                        // refill the stage once this MMA has read it
-                    if (!wait_idle(bar(BAR_VE + st), ph, abort_flag)) { fail(2); break; }
+                    if (!wait64(bar(BAR_VE + st), ph, abort_flag)) { fail(2); break; }
                     load_v(jt + 2);
                 }
             }
