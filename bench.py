@@ -439,11 +439,14 @@ def main():
         pq, pk, pv = qh.pin_memory(), kh.pin_memory(), vh.pin_memory()
         dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
         # One problem per (batch, pair of KV head groups): its Q/K/V slices are contiguous, so each goes through
-        # hifa4_attention_fwd_raw on its own, and three streams keep the host-to-device copy of one
-        # slice, the kernels of another and the device-to-host copy of a third in flight together.
+        # hifa4_attention_fwd_raw on its own; one stream carries all host-to-device copies, one all device-to-host
+        # copies and three the kernels, tied together by events, so that the copy of one slice, the kernels of
+        # another and the read-back of a third are in flight together.  (Finer slices are bound by the host: each
+        # slice costs about a dozen Python-level API calls.)
         G = cfg.Hq // cfg.Hkv
         GPS = 2 if cfg.Hkv % 2 == 0 else 1                               # KV head groups per slice
         streams = [torch.cuda.Stream(device=dev) for _ in range(3)]
+        h2d_stream, d2h_stream = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
         ws_bytes = hb.attention_raw_workspace_bytes(1, G * GPS, GPS, cfg.N, cfg.d, dt, cfg.causal, cfg.Bc)
         ws_s = [torch.empty(ws_bytes, dtype=torch.uint8, device=dev) for _ in streams]
         slices = [(bb, g) for bb in range(cfg.B) for g in range(0, cfg.Hkv, GPS)]
@@ -451,11 +454,11 @@ def main():
         def fork():
             e = torch.cuda.Event()
             e.record()
-            for st_i in streams:
+            for st_i in streams + [h2d_stream, d2h_stream]:
                 st_i.wait_event(e)
 
         def join():
-            for st_i in streams:
+            for st_i in streams + [h2d_stream, d2h_stream]:
                 e = torch.cuda.Event()
                 e.record(st_i)
                 torch.cuda.current_stream().wait_event(e)
@@ -468,14 +471,22 @@ def main():
                 for i, (bb, g) in enumerate(slices):
                     st_i = streams[i % len(streams)]
                     hs, gs = slice(g * G, (g + GPS) * G), slice(g, g + GPS)
-                    with torch.cuda.stream(st_i):
+                    with torch.cuda.stream(h2d_stream):
                         dq[bb:bb + 1, hs].copy_(pq[bb:bb + 1, hs], non_blocking=True)
                         dk[bb:bb + 1, gs].copy_(pk[bb:bb + 1, gs], non_blocking=True)
                         dv[bb:bb + 1, gs].copy_(pv[bb:bb + 1, gs], non_blocking=True)
+                        landed = torch.cuda.Event()
+                        landed.record()
+                    st_i.wait_event(landed)
+                    with torch.cuda.stream(st_i):
                         hb.attention_fwd_raw(dq[bb:bb + 1, hs], dk[bb:bb + 1, gs], dv[bb:bb + 1, gs],
                                              None if s is None else s[gs], None if inv_s is None else inv_s[gs],
                                              cfg.causal, Bc=cfg.Bc, out_dtype=out_code, out=d_out[bb:bb + 1, hs],
                                              workspace=ws_s[i % len(streams)], d_status=status)
+                        done = torch.cuda.Event()
+                        done.record()
+                    d2h_stream.wait_event(done)
+                    with torch.cuda.stream(d2h_stream):
                         po[bb:bb + 1, hs].copy_(d_out[bb:bb + 1, hs], non_blocking=True)
 
             fork()
@@ -501,7 +512,7 @@ def main():
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": po.numel() * po.element_size(),
                     "ms_per_step": e_ms / n_e2e, "out_dtype": str(torch_dt).replace("torch.", ""),
                     "how": f"hifa4_attention_fwd_raw per (batch, KV head group) slice, {len(slices)} slices over "
-                           f"{len(streams)} streams, pinned host buffers"}
+                           f"{len(streams)} kernel streams and two copy streams, pinned host buffers"}
 
         e2e_f32 = e2e_run(hb.F32, torch.float32)
         e2e = e2e_run(hb.F16, torch.float16)
