@@ -165,6 +165,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         // The same thread sets the barriers up and starts the first loads at once (Q and two K tiles), so that
         // they are in flight while the rest of the CTA sets itself up.
         int status_now = args.d_status ? *reinterpret_cast<volatile int*>(args.d_status) : 0;
+        tma_prefetch_desc(&tmap_q); tma_prefetch_desc(&tmap_k); tma_prefetch_desc(&tmap_v);
         mbar_init(bar(BAR_Q), 1);
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(bar(BAR_QKGO + s), 5); mbar_init(bar(BAR_KE + s), 1);
@@ -437,8 +438,10 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         // finalize: out = O / l with l rounded to FP16 (line 13); half kq writes channels (d/2)*kq..
         if (ok && wait64(bar(BAR_PV + ((n_tiles - 1) & 1)), (uint32_t)((n_tiles - 1) >> 1) & 1u, abort_flag)) {
             tc_fence_after();
-            uint32_t lr[4];
+            constexpr int NC = D / 2 / 32;                     // 32-column chunks of this thread's channel half
+            uint32_t lr[4], rbuf[2][32];
             tmem_ld4(t_lane + D, lr);
+            tmem_ld32(t_lane + kq * (D / 2), rbuf[0]);         // the next chunk is always in flight under the current one
             tmem_wait_ld();
             const float ell = __uint_as_float(lr[0]);
             const float l16 = f16_round(ell);
@@ -456,10 +459,9 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             // 128-byte lines per instruction instead of 32 pieces of 16 bytes.
             const uint32_t stage = k_s + (uint32_t)warp * 4096u;
 #pragma unroll
-            for (int cc = 0; cc < D / 2 / 32; ++cc) {
-                uint32_t r[32];
-                tmem_ld32(t_lane + kq * (D / 2) + cc * 32, r);
-                tmem_wait_ld();
+            for (int cc = 0; cc < NC; ++cc) {
+                uint32_t (&r)[32] = rbuf[cc & 1];
+                if (cc + 1 < NC) tmem_ld32(t_lane + kq * (D / 2) + (cc + 1) * 32, rbuf[(cc + 1) & 1]);
                 float o[32];
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
@@ -503,6 +505,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
 #pragma unroll
                     for (int i = 0; i < 4; ++i) dst[i] = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
                 }
+                if (cc + 1 < NC) tmem_wait_ld();
             }
         } else if (ok) {
             fail(11);
