@@ -33,12 +33,10 @@ from paper_2607_04302_b200 import synth  # noqa: E402
 METRIC = "4-bit attention prefill TFLOPS on 1 B200; % of dense 4-bit tensor peak"
 UNIT = "TFLOP/s"
 NOMINAL = {"fp4": 9000.0, "fp8": 4500.0, "bf16": 2250.0}      # dense TFLOP/s, context only
-# dram__bytes_read.sum + dram__bytes_write.sum of one attention launch, from the ncu capture
-# summarised in profiles/attention_fwd_ws_C2.md (bytes per launch; None where not captured)
 # executed warp instructions per 32 scores (ncu opcode counters) and DRAM bytes per launch, from the captures
 # summarised in profiles/attention_fwd_ws64_C2.md and profiles/attention_fwd_ws_bc128_C2.md
-NCU_INSTR_PER_WARP_SCORE = {"attention_fwd_ws64_kernel<128>": 15.5}
-NCU_TRAFFIC_BYTES = {("C2-qwen3-8b-4k", 64): 68.70e6, ("C2-qwen3-8b-4k", 128): 67.14e6}
+NCU_INSTR_PER_WARP_SCORE = {"attention_fwd_ws64_kernel<128>": 15.8, "attention_fwd_ws_kernel<4>": 20.8}
+NCU_TRAFFIC_BYTES = {("C2-qwen3-8b-4k", 64): 70.85e6, ("C2-qwen3-8b-4k", 128): 70.31e6}
 # Issue slots the method itself needs per score on this machine (per 32 scores one warp instruction each):
 # exponential 1, scale-subtract FMA 0.5 (packed), FP16 round trip 1.5, row maximum 0.5, subgroup maxima 0.5,
 # shift selection 1.25, scale-and-round 1.5 (packed), BF16 image 0.5, rescale of the history about 0.7,
