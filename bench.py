@@ -248,6 +248,16 @@ def oracle_scales(cfg):
     return cal["s"], cal["inv_s"]
 
 
+def config_dict(cfg, args, world):
+    """The `config` object of the JSON line (the same for both arms, so that they can be matched)."""
+    return {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "N": cfg.N, "d": cfg.d,
+            "causal": cfg.causal, "Br": 128, "Bc": cfg.Bc, "in_dtype": cfg.dtype, "out_dtype": "f32",
+            "p_dtype": "f32 (variant)" if args.p_f32 else "f16", "qmean": bool(args.qmean),
+            "smooth_mode": cfg.smooth_mode, "step": "hifa4_quantize_qkv + hifa4_attention_fwd",
+            "l2": "flushed between steps (256 MiB write, then a 256 MiB read that drains the dirty lines), outside the per-step events",
+            "parallelism": f"replicated batches x{world}"}
+
+
 def run_reference(args, cfg, rank):
     """--impl reference: the CPU oracle, as it stands, on a bounded sample per step."""
     if rank != 0:
@@ -272,7 +282,7 @@ def run_reference(args, cfg, rank):
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-            "data": "synthetic", "config": {"workload": cfg.name, "causal": cfg.causal, "Bc": cfg.Bc},
+            "data": "synthetic", "config": config_dict(cfg, args, int(os.environ.get("WORLD_SIZE", "1"))),
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -651,12 +661,7 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": cfg.name, "B": cfg.B, "Hq": cfg.Hq, "Hkv": cfg.Hkv, "N": cfg.N, "d": cfg.d,
-                       "causal": cfg.causal, "Br": 128, "Bc": cfg.Bc, "in_dtype": cfg.dtype, "out_dtype": "f32",
-                       "p_dtype": "f32 (variant)" if args.p_f32 else "f16", "qmean": bool(args.qmean),
-                       "smooth_mode": cfg.smooth_mode, "step": "hifa4_quantize_qkv + hifa4_attention_fwd",
-                       "l2": "flushed between steps (256 MiB write, then a 256 MiB read that drains the dirty lines), outside the per-step events",
-                       "parallelism": f"replicated batches x{world}"},
+            "config": config_dict(cfg, args, world),
             "frac_of_nominal_peak": {k_: value / world / v_ for k_, v_ in NOMINAL.items()},
             "clocks": clocks, "e2e": e2e, "e2e_f32_out": e2e_f32, "gpu_launches": launches, "roofline": roofline,
             "roofline_alu": roofline_alu, "quantize": quant, "cpu_baseline": cpu, "context": context,
