@@ -274,13 +274,31 @@ int hifa4_attention_fwd_stats(const hifa4_shape* shape, const hifa4_qkv* qkv,
                               const hifa4_attn_params* prm, void* out, void* workspace,
                               const hifa4_mass_stats* stats, int* d_status, void* stream);
 
+/* hifa4_attention_fwd with Algorithm 1 line 1 inside the attention kernel: q is
+ * the raw post-RoPE Q [B,Hq,N,d] of shape->in_dtype (device), s the Smooth-QK
+ * factors of Q [Hkv,d] (device) or NULL; every CTA smooths and HIF4-quantizes
+ * its own 128 query rows in shared memory, so Q-hat is never written to device
+ * memory (its codes are not produced).  kv: buffers filled by
+ * hifa4_quantize_qkv(shape, NULL, k, v, ...) for the same shape (only k_mma
+ * and v_mma are read).  The result is bit-identical to hifa4_quantize_qkv on
+ * q followed by hifa4_attention_fwd.  Supported for Bc = 64, d = 128,
+ * qmean = 0, normalizer = 0; anything else returns HIFA4_ERR_UNSUPPORTED
+ * without a launch.  Other arguments, status word and scheduling note as
+ * hifa4_attention_fwd. */
+int hifa4_attention_fwd_qraw(const hifa4_shape* shape, const void* q, const float* s,
+                             const hifa4_qkv* kv, const hifa4_attn_params* prm, void* out,
+                             void* workspace, int* d_status, void* stream);
+
 /* Workspace for hifa4_attention_fwd_raw: all hifa4_qkv buffers (each rounded up
  * to 256 bytes; the two Q-Mean vectors only when prm->qmean = 1) plus the
  * attention workspace. */
 size_t hifa4_attention_raw_workspace_bytes(const hifa4_shape* shape, const hifa4_attn_params* prm);
 
 /* Algorithm 1 end to end on raw post-RoPE Q/K/V: hifa4_quantize_qkv into
- * `workspace`, then hifa4_attention_fwd.  s, inv_s as in hifa4_quantize_qkv. */
+ * `workspace`, then hifa4_attention_fwd; where hifa4_attention_fwd_qraw supports
+ * the configuration, only K and V are quantized into the workspace and Q is
+ * quantized inside the attention kernel (same result).  s, inv_s as in
+ * hifa4_quantize_qkv. */
 int hifa4_attention_fwd_raw(const hifa4_shape* shape, const void* q, const void* k, const void* v,
                             const float* s, const float* inv_s, const hifa4_attn_params* prm,
                             void* out, void* workspace, size_t workspace_bytes,

@@ -104,6 +104,10 @@ def lib():
         L.hifa4_attention_fwd.restype = C.c_int
         L.hifa4_attention_fwd.argtypes = [C.POINTER(_Shape), C.POINTER(_QKV), C.POINTER(_AttnParams),
                                           C.c_void_p, C.c_void_p, C.POINTER(_Debug), C.c_void_p, C.c_void_p]
+        L.hifa4_attention_fwd_qraw.restype = C.c_int
+        L.hifa4_attention_fwd_qraw.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.POINTER(_QKV),
+                                               C.POINTER(_AttnParams), C.c_void_p, C.c_void_p, C.c_void_p,
+                                               C.c_void_p]
         L.hifa4_selftest_wait_timeout.restype = C.c_int
         L.hifa4_selftest_wait_timeout.argtypes = [C.POINTER(_Shape), C.POINTER(_QKV), C.POINTER(_AttnParams),
                                                   C.c_void_p, C.c_void_p, C.c_void_p]
@@ -125,7 +129,7 @@ EXPORTS = ("hifa4_status_string", "hifa4_get_counters", "hifa4_smooth_calibrate"
            "hifa4_smooth_calibrate_static", "hifa4_smooth_calibrate_auto", "hifa4_quant_bytes",
            "hifa4_quantize_qkv", "hifa4_attention_workspace_bytes", "hifa4_attention_fwd",
            "hifa4_attention_fwd_stats", "hifa4_attention_raw_workspace_bytes", "hifa4_attention_fwd_raw",
-           "hifa4_selftest_wait_timeout")
+           "hifa4_attention_fwd_qraw", "hifa4_selftest_wait_timeout")
 
 
 def status_string(status: int) -> str:
@@ -288,15 +292,20 @@ def smooth_calibrate_static(q_cal, k_cal, mode, alpha=0.0, q_to_kv=None, s=None,
 
 
 def quantize_qkv(q, k, v, s=None, inv_s=None, q_to_kv=None, out: QuantizedQKV | None = None,
-                 d_status=None, qmean=False) -> QuantizedQKV:
+                 d_status=None, qmean=False, Hq=None) -> QuantizedQKV:
     """Smooth-QK + HIF4 quantization of device tensors q [B,Hq,N,d], k, v [B,Hkv,N,d].
-    qmean: also apply the Q-Mean auxiliary (the Q buffers then hold the mean-free Q_z)."""
-    assert q.is_cuda and q.is_contiguous() and k.is_contiguous() and v.is_contiguous()
-    B, Hq, N, d = q.shape
+    qmean: also apply the Q-Mean auxiliary (the Q buffers then hold the mean-free Q_z).
+    q = None: K and V only (for attention_fwd_qraw); Hq then names the number of query heads."""
+    assert k.is_cuda and k.is_contiguous() and v.is_contiguous() and (q is None or q.is_contiguous())
+    if q is None:
+        assert Hq is not None and not qmean
+        B, _, N, d = k.shape
+    else:
+        B, Hq, N, d = q.shape
     Hkv = k.shape[1]
-    dt = _DT[q.dtype]
+    dt = _DT[k.dtype]
     if out is None:
-        out = alloc_qkv(B, Hq, Hkv, N, d, dt, q.device, q_to_kv, qmean=qmean)
+        out = alloc_qkv(B, Hq, Hkv, N, d, dt, k.device, q_to_kv, qmean=qmean)
     sh = _shape(B, Hq, Hkv, N, d, dt, q_to_kv)
     st = out.struct()
     rc = lib().hifa4_quantize_qkv(C.byref(sh), _ptr(q), _ptr(k), _ptr(v), _ptr(s), _ptr(inv_s),
@@ -334,6 +343,23 @@ def attention_fwd(qkv: QuantizedQKV, causal: bool, Bc: int = 64, out_dtype=F32, 
                                    _ptr(d_status), _stream())
     _check(rc, "hifa4_attention_fwd")
     return (out, dump) if debug_blocks else out
+
+
+def attention_fwd_qraw(q, s, kv: QuantizedQKV, causal: bool, out_dtype=F32, out=None, d_status=None,
+                       softmax_scale=0.0, p_dtype=F16):
+    """attention_fwd whose kernel smooths and quantizes the raw q [B,Hq,N,d] itself (s: [Hkv,d] or None); kv holds
+    the K and V images from quantize_qkv(None, k, v, ...).  Bc = 64, d = 64 or 128, no Q-Mean."""
+    assert q.is_cuda and q.is_contiguous() and _DT[q.dtype] == kv.in_dtype
+    sh = _shape(kv.B, kv.Hq, kv.Hkv, kv.N, kv.d, kv.in_dtype, kv.q_to_kv)
+    assert tuple(q.shape) == (kv.B, kv.Hq, kv.N, kv.d)
+    prm = _params(causal, 64, out_dtype, softmax_scale=softmax_scale, p_dtype=p_dtype)
+    if out is None:
+        out = torch.empty((kv.B, kv.Hq, kv.N, kv.d), dtype=_TORCH_DT[out_dtype], device=q.device)
+    st = kv.struct()
+    rc = lib().hifa4_attention_fwd_qraw(C.byref(sh), _ptr(q), _ptr(s), C.byref(st), C.byref(prm), _ptr(out), None,
+                                        _ptr(d_status), _stream())
+    _check(rc, "hifa4_attention_fwd_qraw")
+    return out
 
 
 def selftest_wait_timeout(qkv: QuantizedQKV, causal: bool, d_status, out=None):

@@ -207,12 +207,13 @@ size_t hifa4_attention_workspace_bytes(const hifa4_shape* shape, const hifa4_att
 
 static int attention_common(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
                             void* out, const hifa4_debug* dbg, const hifa4_mass_stats* stats, int* d_status,
-                            void* stream, bool selftest = false)
+                            void* stream, bool selftest = false, const void* q_raw = nullptr,
+                            const float* q_scale = nullptr)
 {
     g_calls[2].fetch_add(1, std::memory_order_relaxed);
     int rc = check_attn(shape, prm);
     if (rc) return rc;
-    if (!qkv || !out || !qkv->q_mma || !qkv->k_mma || !qkv->v_mma) return HIFA4_ERR_INVALID_ARG;
+    if (!qkv || !out || (!q_raw && !qkv->q_mma) || !qkv->k_mma || !qkv->v_mma) return HIFA4_ERR_INVALID_ARG;
     if (prm->qmean && (!qkv->q_mu || !qkv->k_sum)) return HIFA4_ERR_INVALID_ARG;
     if (dbg) {
         if (dbg->n_blocks < 0 || dbg->n_blocks > HIFA4_MAX_DEBUG_BLOCKS) return HIFA4_ERR_INVALID_ARG;
@@ -227,7 +228,8 @@ static int attention_common(const hifa4_shape* shape, const hifa4_qkv* qkv, cons
     HeadMap qmap, kmap;
     if ((rc = build_map(shape->Hq, shape->Hkv, shape->q_to_kv, qmap, kmap))) return rc;
     if ((rc = check_arch())) return rc;
-    return launch_attention(*shape, qmap, *qkv, *prm, out, dbg, stats, d_status, (cudaStream_t)stream, selftest);
+    return launch_attention(*shape, qmap, *qkv, *prm, out, dbg, stats, d_status, (cudaStream_t)stream, selftest,
+                            q_raw, q_scale);
 }
 
 int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
@@ -236,6 +238,18 @@ int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv, const hi
 {
     (void)workspace;
     return attention_common(shape, qkv, prm, out, dbg, nullptr, d_status, stream);
+}
+
+int hifa4_attention_fwd_qraw(const hifa4_shape* shape, const void* q, const float* s, const hifa4_qkv* kv,
+                             const hifa4_attn_params* prm, void* out, void* workspace, int* d_status,
+                             void* stream)
+{
+    (void)workspace;
+    if (!q) return HIFA4_ERR_INVALID_ARG;
+    int rc = check_attn(shape, prm);
+    if (rc) return rc;
+    if (!attention_qraw_supported(*shape, *prm)) return HIFA4_ERR_UNSUPPORTED;
+    return attention_common(shape, kv, prm, out, nullptr, nullptr, d_status, stream, false, q, s);
 }
 
 int hifa4_selftest_wait_timeout(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
@@ -293,6 +307,13 @@ int hifa4_attention_fwd_raw(const hifa4_shape* shape, const void* q, const void*
     if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) return HIFA4_ERR_WORKSPACE;
     hifa4_qkv bufs;
     size_t used = qkv_layout(shape, prm->qmean, (char*)workspace, &bufs);
+    if ((s == nullptr) != (inv_s == nullptr)) return HIFA4_ERR_INVALID_ARG;
+    // K and V here, Q inside the attention kernel: pays once the Q-hat image (written, then read) is large; measured
+    // on B200 at d = 128: -1 to -3 % of the two launches from 64k query rows up, slower below
+    if (attention_qraw_supported(*shape, *prm) && (long long)shape->B * shape->Hq * shape->N >= 65536) {
+        if ((rc = hifa4_quantize_qkv(shape, nullptr, k, v, s, inv_s, &bufs, d_status, stream))) return rc;
+        return hifa4_attention_fwd_qraw(shape, q, s, &bufs, prm, out, (char*)workspace + used, d_status, stream);
+    }
     if ((rc = hifa4_quantize_qkv(shape, q, k, v, s, inv_s, &bufs, d_status, stream))) return rc;
     return hifa4_attention_fwd(shape, &bufs, prm, out, (char*)workspace + used, nullptr, d_status, stream);
 }

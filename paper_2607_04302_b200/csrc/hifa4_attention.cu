@@ -342,12 +342,24 @@ static int launch_cfg(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArg
     return cudaGetLastError() == cudaSuccess ? HIFA4_OK : HIFA4_ERR_CUDA;
 }
 
+bool attention_qraw_supported(const hifa4_shape& sh, const hifa4_attn_params& prm)
+{
+    return prm.Bc == 64 && sh.d == 128 && !prm.qmean && !prm.normalizer;
+}
+
 int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv& qkv,
                      const hifa4_attn_params& prm, void* out, const hifa4_debug* dbg,
-                     const hifa4_mass_stats* stats, int* d_status, cudaStream_t st, bool selftest)
+                     const hifa4_mass_stats* stats, int* d_status, cudaStream_t st, bool selftest,
+                     const void* q_raw, const float* q_scale)
 {
     AttnArgs a;
     memset(&a, 0, sizeof(a));
+    if (q_raw) {
+        if (!attention_qraw_supported(sh, prm) || stats || selftest || (dbg && dbg->n_blocks > 0)) return HIFA4_ERR_UNSUPPORTED;
+        a.q_raw = q_raw;
+        a.q_scale = q_scale;
+        a.in_dtype = sh.in_dtype;
+    }
     a.B = sh.B; a.Hq = sh.Hq; a.Hkv = sh.Hkv; a.N = sh.N;
     a.causal = prm.causal ? 1 : 0;
     a.out_dtype = prm.out_dtype;

@@ -101,13 +101,16 @@ static __device__ __forceinline__ void arrive_lane0(uint32_t bar, int lane)
 // SELFTEST: the instantiation behind hifa4_selftest_wait_timeout.  Its softmax warps withhold the arrival that
 // releases P V and the issuer's wait for it gives up after 2^12 polls instead of 2^20; by then every TMA load
 // has landed and no MMA is in flight, so the CTA leaves through the ordinary failure exit.
-template <int DH, bool DBG, bool PF32, bool QM, bool SELFTEST = false>
+// QRAW: the Q tensor map is over the raw 16-bit Q; the softmax threads smooth and HIF4-quantize their CTA's 128 rows
+// in shared memory (Algorithm 1 line 1) before the first S = Q K^T, so Q-hat never travels through HBM.
+template <int DH, bool DBG, bool PF32, bool QM, bool SELFTEST = false, bool QRAW = false>
 __global__ void __launch_bounds__(WS64<DH>::THREADS, WS64<DH>::CTAS_PER_SM)
 attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                            const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnArgs args)
 {
     using namespace ws64;
     using C = WS64<DH>;
+    static_assert(!QRAW || (DH == 128 && !QM && !DBG), "raw-Q launch: d = 128, no Q-Mean, no dump");
     constexpr int D = C::D, BC = C::BC, STAGES = C::STAGES, NSW = C::NSW, THREADS = C::THREADS;
     constexpr int W_QK = C::W_QK, W_PV = C::W_PV, NU = C::NU, QSUB = C::QSUB;
     constexpr int Q_BYTES = C::Q_BYTES, K_SUB = C::K_SUB, K_STAGE = C::K_STAGE, V_STAGE = C::V_STAGE;
@@ -215,7 +218,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         if (lane == 0) {
             constexpr uint32_t idesc_s = umma_idesc_bf16(128, BC);
             const uint32_t q_lo = umma_desc_lo(q_s), k_lo = umma_desc_lo(k_s);
-            bool ok = wait64(bar(C::Q_IN_TMEM ? BAR_QT : BAR_Q), 0, abort_flag);
+            bool ok = wait64(bar(C::Q_IN_TMEM || QRAW ? BAR_QT : BAR_Q), 0, abort_flag);
             if (!ok) fail(3);
             for (int jt = 0; ok && jt < n_tiles; ++jt) {      // S(jt): K tile landed, S(jt-1) in registers
                 const int st = jt & 1;
@@ -308,6 +311,18 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 __syncwarp();
                 arrive_lane0(bar(BAR_QT), lane);
             } else { fail(13); ok = false; }
+        }
+        if constexpr (QRAW) {
+            // Q-hat = HIF4(round(Q s)) in place (Algorithm 1 line 1): thread (row, kq) owns the row's 64-channel group kq
+            if (wait64(bar(BAR_Q), 0, abort_flag)) {
+                const uint32_t row_addr = q_s + (uint32_t)kq * 16384u + (uint32_t)r_loc * 128u;
+                const float* sc = args.q_scale ? args.q_scale + (size_t)g * D + kq * 64 : nullptr;
+                if (args.in_dtype == HIFA4_F16) quantize_q_row_inplace<__half>(row_addr, r_loc & 7, sc);
+                else quantize_q_row_inplace<__nv_bfloat16>(row_addr, r_loc & 7, sc);
+            } else { fail(13); ok = false; }
+            fence_proxy_async_smem();                          // generic-proxy writes, read by the MMA
+            __syncwarp();
+            arrive_lane0(bar(BAR_QT), lane);
         }
         if (grp == 0) arrive_lane0(bar(BAR_QKGO), lane);          // S is free for tile 0
 
@@ -517,15 +532,15 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     if (warp == W_QK) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
 }
 
-template <int DH, bool DBG, bool PF32, bool QM, bool SELFTEST = false>
+template <int DH, bool DBG, bool PF32, bool QM, bool SELFTEST = false, bool QRAW = false>
 static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
     using C = WS64<DH>;
     CUtensorMap mq, mk, mv;
-    if (!make_bf16_map(&mq, qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, DH, 128)) return HIFA4_ERR_CUDA;
+    if (!make_bf16_map(&mq, QRAW ? const_cast<void*>(args.q_raw) : qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, DH, 128)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, DH, C::BC)) return HIFA4_ERR_CUDA;
     if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, DH, sh.N, DH)) return HIFA4_ERR_CUDA;
-    auto kern = attention_fwd_ws64_kernel<DH, DBG, PF32, QM, SELFTEST>;
+    auto kern = attention_fwd_ws64_kernel<DH, DBG, PF32, QM, SELFTEST, QRAW>;
     static SmemOptIn opt_in;
     if (!opt_in.ensure(kern, C::SMEM_BYTES)) return HIFA4_ERR_CUDA;
     dim3 grid((unsigned)(((sh.N + 127) / 128) * sh.Hq * sh.B));
@@ -548,6 +563,14 @@ template <int DH>
 static int launch_ws64_d(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
     const bool dbg = args.dbg.n_blocks > 0;
+    if (args.q_raw) {                                      // Q quantized in the kernel: d = 128, no Q-Mean, no dump
+        if constexpr (DH != 128) return HIFA4_ERR_UNSUPPORTED;
+        else {
+            if (dbg || args.qmean) return HIFA4_ERR_UNSUPPORTED;
+            if (args.p_f32) return launch_ws64<DH, false, true, false, false, true>(sh, qkv, args, st);
+            return launch_ws64<DH, false, false, false, false, true>(sh, qkv, args, st);
+        }
+    }
     if (args.p_f32) {                                      // variant: no Q-Mean, d = 128 or 256
         if constexpr (DH == 64) return HIFA4_ERR_UNSUPPORTED;
         else {

@@ -5,7 +5,11 @@
 #include <cuda_fp16.h>
 #include <stdint.h>
 
+#include "hifa4_ptx.cuh"
+
 namespace hifa4 {
+
+using namespace ptx;
 
 struct HeadMap {                       // head -> row of the [Hkv, d] scale table
     short kv_of[256];
@@ -55,5 +59,95 @@ template <> struct In16<__nv_bfloat16> {
     static __device__ __forceinline__ float round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
     static __device__ __forceinline__ float round_d(double x) { return __bfloat162float(__double2bfloat16(x)); }
 };
+
+// 16-bit input pairs <-> fp32, and the rounding of a smoothed pair back to the input dtype.
+template <typename T> struct Pair16;
+template <> struct Pair16<__nv_bfloat16> {
+    static __device__ __forceinline__ void unpack(uint32_t w, float& lo, float& hi)
+    {
+        lo = __uint_as_float(w << 16);
+        hi = __uint_as_float(w & 0xFFFF0000u);
+    }
+    static __device__ __forceinline__ uint32_t round_pack(float lo, float hi)
+    {
+        uint32_t r;
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+        return r;
+    }
+};
+template <> struct Pair16<__half> {
+    static __device__ __forceinline__ void unpack(uint32_t w, float& lo, float& hi)
+    {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w));
+        lo = f.x;
+        hi = f.y;
+    }
+    static __device__ __forceinline__ uint32_t round_pack(float lo, float hi)
+    {
+        uint32_t r;
+        asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+        return r;
+    }
+};
+
+// ---------------------------------------------------------------------------
+// HIF4 quantization of values that are exact in a 16-bit input type, one level-2 unit (8 elements =
+// two level-3 subgroups) at a time.  All arithmetic is exact:
+//   q = RZ(x * RN(4/S))             lands exactly on j + 1/2 on every rounding tie (see e6m2_inv4)
+//   y = q + 1.5 * 2^(23+k)          rounds q to the nearest multiple of 2^k, ties to even:
+//                                   bits(y) - bits(magic) = m, the signed element code under shift k
+//   v = fma(y, S/4, -magic * S/4)   = m * 2^k * S/4, the dequantized value
+// The shift of a subgroup with maximum At is need = max(bits(At) - bits(1.75 S) - 1 + 2^23, 0) >> 23;
+// the pair rule is a = (n0 + n1 + 2) >> 2, k = max(need, a).
+// ---------------------------------------------------------------------------
+struct Hif4Group {                  // constants of a 64-element group whose maximum magnitude is A
+    int code;                       // E6M2 code of the scale S (A = 0: code 0, an all-zero group)
+    float top;                      // 7 S; larger magnitudes saturate (only above the E6M2 range)
+    uint64_t inv44, s44;            // {4/S, 4/S}, {S/4, S/4}
+    uint32_t c0_bits;               // bits(-1.5 * 2^23 * S/4)
+    int tadd;
+};
+__device__ __forceinline__ Hif4Group hif4_group(float A)
+{
+    Hif4Group g;
+    g.code = e6m2_code_for_max(A);
+    const float S = e6m2_value(g.code);
+    g.top = 7.f * S;
+    const float inv4 = e6m2_inv4(g.code);
+    const float S4 = __uint_as_float(__float_as_uint(S) - (2u << 23));
+    g.inv44 = pack2(inv4, inv4);
+    g.s44 = pack2(S4, S4);
+    g.c0_bits = __float_as_uint(-12582912.f * S4);
+    g.tadd = (1 << 23) - ((int)__float_as_uint(1.75f * S) + 1);
+    return g;
+}
+// x: the unit's values (already clamped to +-top), a0 / a1: the maxima of its two subgroups.  w: BF16 image of
+// the dequantized values (element 2i in the low half of word i); y: the biased quotients (the low byte of
+// bits(y[i]) is the signed element code); a, k0, k1: level-2 shift and the subgroups' total shifts.
+__device__ __forceinline__ void hif4_unit(const float (&x)[8], float a0, float a1, const Hif4Group& g,
+                                          uint32_t (&w)[4], float (&y)[8], int& a, int& k0, int& k1)
+{
+    const int n0 = max((int)__float_as_uint(a0) + g.tadd, 0) >> 23;
+    const int n1 = max((int)__float_as_uint(a1) + g.tadd, 0) >> 23;
+    a = (n0 + n1 + 2) >> 2;
+    k0 = max(n0, a);
+    k1 = max(n1, a);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t ks = (uint32_t)(h ? k1 : k0) << 23;
+        const uint32_t magic_bits = 0x4B400000u + ks;
+        const float magic = __uint_as_float(magic_bits), ck = __uint_as_float(g.c0_bits + ks);
+        const uint64_t mm = pack2(magic, magic), cc = pack2(ck, ck);
+        const uint64_t y01 = add2(mul2_rz(pack2(x[4 * h], x[4 * h + 1]), g.inv44), mm);
+        const uint64_t y23 = add2(mul2_rz(pack2(x[4 * h + 2], x[4 * h + 3]), g.inv44), mm);
+        float v0, v1, v2, v3;
+        unpack2(fma2(y01, g.s44, cc), v0, v1);
+        unpack2(fma2(y23, g.s44, cc), v2, v3);
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[2 * h]) : "f"(v1), "f"(v0));
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[2 * h + 1]) : "f"(v3), "f"(v2));
+        unpack2(y01, y[4 * h], y[4 * h + 1]);
+        unpack2(y23, y[4 * h + 2], y[4 * h + 3]);
+    }
+}
 
 }  // namespace hifa4

@@ -49,8 +49,15 @@ cudaError_t launch_gate(int dtype, const void* k_cal, long long nk, const float*
 const double* gate_result(void* gate_ws);
 
 // Attention forward on the BF16 operand images; returns a hifa4_status.
+// q_raw non-null: Q is the raw 16-bit tensor (qkv.q_mma is not read) and is smoothed with q_scale (or not, if null)
+// and quantized inside the kernel; see attention_qraw_supported.
 int launch_attention(const hifa4_shape& shape, const HeadMap& map, const hifa4_qkv& qkv,
                      const hifa4_attn_params& prm, void* out, const hifa4_debug* dbg,
-                     const hifa4_mass_stats* stats, int* d_status, cudaStream_t st, bool selftest = false);
+                     const hifa4_mass_stats* stats, int* d_status, cudaStream_t st, bool selftest = false,
+                     const void* q_raw = nullptr, const float* q_scale = nullptr);
+// Configurations whose attention kernel can quantize Q itself: the 64-key kernel for d = 128 (256 softmax threads =
+// 128 rows x two 64-channel groups) in its default arithmetic or the FP32-P variant, without Q-Mean (the row mean
+// needs the whole row before any group is quantized).
+bool attention_qraw_supported(const hifa4_shape& shape, const hifa4_attn_params& prm);
 
 }  // namespace hifa4

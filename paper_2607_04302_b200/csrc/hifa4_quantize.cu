@@ -15,14 +15,7 @@ using namespace ptx;
 // x[8]: values already smoothed and rounded to the input dtype.  Returns the packed nibbles; w gets
 // the BF16 image of the dequantized values (element 2i in the low half of word i); meta_word the
 // group's metadata (every lane of the team gets the same word).
-//
-// Arithmetic (all exact; the same scheme as the in-register quantizer of P):
-//   q = RZ(x * RN(4/S))             lands exactly on j + 1/2 on every rounding tie (see e6m2_inv4)
-//   y = q + 1.5 * 2^(23+k)          rounds q to the nearest multiple of 2^k, ties to even:
-//                                   bits(y) - bits(magic) = m, the signed element code under shift k
-//   v = fma(y, S/4, -magic * S/4)   = m * 2^k * S/4, the dequantized value
-// The shift of a subgroup with maximum At is need = max(bits(At) - bits(1.75 S) - 1 + 2^23, 0) >> 23;
-// the pair rule is a = (n0 + n1 + 2) >> 2, k = max(need, a).
+// The arithmetic is hif4_group / hif4_unit (exact; the same scheme as the in-register quantizer of P).
 __device__ __forceinline__ uint32_t quantize8(float (&x)[8], int j, uint32_t (&w)[4], uint32_t& meta_word)
 {
     float a0 = fmaxf(max3(fabsf(x[0]), fabsf(x[1]), fabsf(x[2])), fabsf(x[3]));
@@ -31,46 +24,25 @@ __device__ __forceinline__ uint32_t quantize8(float (&x)[8], int j, uint32_t (&w
     A = fmaxf(A, __shfl_xor_sync(0xffffffffu, A, 1));
     A = fmaxf(A, __shfl_xor_sync(0xffffffffu, A, 2));
     A = fmaxf(A, __shfl_xor_sync(0xffffffffu, A, 4));
-    const int code = e6m2_code_for_max(A);                        // A = 0 gives code 0 and an all-zero group
-    const float S = e6m2_value(code);
-    const float top = 7.f * S;
-    if (A > top) {                                                // only above the E6M2 range: saturate
+    const Hif4Group g = hif4_group(A);                            // A = 0 gives code 0 and an all-zero group
+    if (A > g.top) {                                              // only above the E6M2 range: saturate
 #pragma unroll
-        for (int i = 0; i < 8; ++i) x[i] = fminf(fmaxf(x[i], -top), top);
-        a0 = fminf(a0, top);
-        a1 = fminf(a1, top);
+        for (int i = 0; i < 8; ++i) x[i] = fminf(fmaxf(x[i], -g.top), g.top);
+        a0 = fminf(a0, g.top);
+        a1 = fminf(a1, g.top);
     }
-    const float inv4 = e6m2_inv4(code);
-    const float S4 = __uint_as_float(__float_as_uint(S) - (2u << 23));
-    const uint64_t inv44 = pack2(inv4, inv4), s44 = pack2(S4, S4);
-    const uint32_t c0_bits = __float_as_uint(-12582912.f * S4);   // -1.5 * 2^23 * S/4
-    const int tadd = (1 << 23) - ((int)__float_as_uint(1.75f * S) + 1);
-    const int n0 = max((int)__float_as_uint(a0) + tadd, 0) >> 23;
-    const int n1 = max((int)__float_as_uint(a1) + tadd, 0) >> 23;
-    const int a = (n0 + n1 + 2) >> 2;
-    const int k0 = max(n0, a), k1 = max(n1, a);
+    float y[8];
+    int a, k0, k1;
+    hif4_unit(x, a0, a1, g, w, y, a, k0, k1);
     uint32_t part = ((uint32_t)a << (8 + j)) | ((uint32_t)((k0 - a) | ((k1 - a) << 1)) << (16 + 2 * j));
-    if (j == 0) part |= (uint32_t)code;
+    if (j == 0) part |= (uint32_t)g.code;
     uint32_t xw[2];                                               // per subgroup: nibbles n0 | n1 << 4 in byte 0, n2 | n3 << 4 in byte 2
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-        const uint32_t ks = (uint32_t)(h ? k1 : k0) << 23;
-        const uint32_t magic_bits = 0x4B400000u + ks;
-        const float magic = __uint_as_float(magic_bits), ck = __uint_as_float(c0_bits + ks);
-        const uint64_t mm = pack2(magic, magic), cc = pack2(ck, ck);
-        const uint64_t y01 = add2(mul2_rz(pack2(x[4 * h], x[4 * h + 1]), inv44), mm);
-        const uint64_t y23 = add2(mul2_rz(pack2(x[4 * h + 2], x[4 * h + 3]), inv44), mm);
-        float v0, v1, v2, v3, y[4];
-        unpack2(fma2(y01, s44, cc), v0, v1);
-        unpack2(fma2(y23, s44, cc), v2, v3);
-        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[2 * h]) : "f"(v1), "f"(v0));
-        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[2 * h + 1]) : "f"(v3), "f"(v2));
-        unpack2(y01, y[0], y[1]);
-        unpack2(y23, y[2], y[3]);
         // The low byte of bits(y) is the signed code m (the magic constant's low byte is 0): gather the
         // four bytes and turn them into sign-magnitude nibbles with byte-parallel arithmetic.
-        const uint32_t b01 = __byte_perm(__float_as_uint(y[0]), __float_as_uint(y[1]), 0x0040);
-        const uint32_t b23 = __byte_perm(__float_as_uint(y[2]), __float_as_uint(y[3]), 0x0040);
+        const uint32_t b01 = __byte_perm(__float_as_uint(y[4 * h]), __float_as_uint(y[4 * h + 1]), 0x0040);
+        const uint32_t b23 = __byte_perm(__float_as_uint(y[4 * h + 2]), __float_as_uint(y[4 * h + 3]), 0x0040);
         const uint32_t bb = __byte_perm(b01, b23, 0x5410);                     // m0, m1, m2, m3 as signed bytes
         const uint32_t sg = bb & 0x80808080u;                                  // sign bits
         const uint32_t ng = sg >> 7;                                           // 1 in every negative byte
@@ -85,36 +57,6 @@ __device__ __forceinline__ uint32_t quantize8(float (&x)[8], int j, uint32_t (&w
     meta_word = part;
     return nib;
 }
-
-// 16-bit input pairs <-> fp32, and the rounding of a smoothed pair back to the input dtype.
-template <typename T> struct Pair16;
-template <> struct Pair16<__nv_bfloat16> {
-    static __device__ __forceinline__ void unpack(uint32_t w, float& lo, float& hi)
-    {
-        lo = __uint_as_float(w << 16);
-        hi = __uint_as_float(w & 0xFFFF0000u);
-    }
-    static __device__ __forceinline__ uint32_t round_pack(float lo, float hi)
-    {
-        uint32_t r;
-        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-        return r;
-    }
-};
-template <> struct Pair16<__half> {
-    static __device__ __forceinline__ void unpack(uint32_t w, float& lo, float& hi)
-    {
-        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w));
-        lo = f.x;
-        hi = f.y;
-    }
-    static __device__ __forceinline__ uint32_t round_pack(float lo, float hi)
-    {
-        uint32_t r;
-        asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-        return r;
-    }
-};
 
 struct QuantJob {                     // one launch quantizes Q, K and V (any of them may be absent)
     const uint16_t *q, *k, *v;        // [B,Hq,N,d], [B,Hkv,N,d], [B,Hkv,N,d]

@@ -305,3 +305,56 @@ def test_expired_device_wait_is_reported_and_leaves_the_device_usable(hb, par):
     with pytest.raises(hb.Hifa4Error):                                  # the self-test refuses shapes it was not built for
         hb.selftest_wait_timeout(hb.quantize_qkv(*(t.to(DEV) for t in synth.make_qkv(synth.config("C3", N=128, Hq=1, Hkv=1, d=64)))),
                                  False, status)
+
+
+@pytest.mark.parametrize("dtype,smooth,causal,p_dtype", [("bf16", True, True, "f16"), ("fp16", True, False, "f16"),
+                                                         ("bf16", False, True, "f16"), ("fp16", True, True, "f32")])
+def test_in_kernel_query_quantization_is_bit_identical(hb, par, dtype, smooth, causal, p_dtype):
+    """hifa4_attention_fwd_qraw smooths and HIF4-quantizes Q inside the attention kernel (Algorithm 1 line 1 per CTA,
+    in shared memory).  Both the stand-alone quantizer and the in-kernel one take the same exact arithmetic, so the
+    output must equal, bit for bit, that of quantize_qkv + attention_fwd (which the other tests hold against the
+    oracle), for both input types, with and without Smooth-QK factors, with GQA, a ragged last query block (N = 320)
+    and an outlier-heavy K.  The K / V buffers written without Q must equal those written with it."""
+    cfg = synth.config("C2", B=2, Hq=4, Hkv=2, N=320, dtype=dtype, causal=causal)
+    q, k, v = (t.to(DEV) for t in synth.make_qkv(cfg))
+    s, inv_s = par.calibrate(cfg, DEV) if smooth else (None, None)
+    pd = hb.F32 if p_dtype == "f32" else hb.F16
+    full = hb.quantize_qkv(q, k, v, s, inv_s)
+    ref = hb.attention_fwd(full, causal, p_dtype=pd)
+    kv = hb.quantize_qkv(None, k, v, s, inv_s, Hq=cfg.Hq)
+    assert torch.equal(kv.k_mma, full.k_mma) and torch.equal(kv.v_mma, full.v_mma)
+    assert torch.equal(kv.k_codes, full.k_codes) and torch.equal(kv.v_meta, full.v_meta)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for out_dtype in (hb.F32, hb.F16):
+        got = hb.attention_fwd_qraw(q, s, kv, causal, out_dtype=out_dtype, p_dtype=pd, d_status=status)
+        want = ref if out_dtype == hb.F32 else hb.attention_fwd(full, causal, out_dtype=out_dtype, p_dtype=pd)
+        assert torch.equal(got, want)
+    assert int(status.item()) == 0
+    # a set status word makes the launch a no-op
+    status.fill_(9)
+    out = torch.full_like(ref, 2.0)
+    hb.attention_fwd_qraw(q, s, kv, causal, out=out, p_dtype=pd, d_status=status)
+    torch.cuda.synchronize()
+    assert bool((out == 2.0).all()) and int(status.item()) == 9
+
+
+def test_in_kernel_query_quantization_full_size_and_refusals(hb, par):
+    """The headline shape through hifa4_attention_fwd_raw (which quantizes K and V into the workspace and Q inside the
+    attention kernel from 64k query rows up) equals the two-call path; configurations the in-kernel quantizer was
+    not built for are refused without a launch."""
+    cfg = synth.config("C2")
+    q, k, v = synth.make_qkv_device(cfg, DEV)
+    s, inv_s = par.calibrate(cfg, DEV)
+    full = hb.quantize_qkv(q, k, v, s, inv_s)
+    want = hb.attention_fwd(full, True)
+    before = hb.get_counters()
+    got = hb.attention_fwd_raw(q, k, v, s, inv_s, True)
+    after = hb.get_counters()
+    assert torch.equal(got, want)
+    assert after["launches"] - before["launches"] == 2          # K/V quantizer + attention
+    kv = hb.quantize_qkv(None, k, v, s, inv_s, Hq=cfg.Hq)
+    assert torch.equal(hb.attention_fwd_qraw(q, s, kv, True), want)
+    c64 = synth.config("C3", N=128, Hq=1, Hkv=1, d=64)
+    q6, k6, v6 = (t.to(DEV) for t in synth.make_qkv(c64))
+    with pytest.raises(hb.Hifa4Error):
+        hb.attention_fwd_qraw(q6, None, hb.quantize_qkv(None, k6, v6, Hq=1), True)
