@@ -169,9 +169,10 @@ def measure_gemm_peaks(dev):
     return res
 
 
-def time_workload(hb, cfg, dev, steps, warmup, flush_l2, s=None, inv_s=None, qmean=False, p_f32=False):
+def time_workload(hb, cfg, dev, steps, warmup, flush_l2, s=None, inv_s=None, qmean=False, p_f32=False, fused_q=False):
     """Device-resident timing of one configuration: per-step time of quantize + attention (events around each
-    step, L2 flushed between steps) and, from a second pass with one more event, the attention launch alone."""
+    step, L2 flushed between steps) and, from a second pass with one more event, the attention launch alone.
+    fused_q: K and V through the quantizer, Q quantized inside the attention kernel (hifa4_attention_fwd_qraw)."""
     q, k, v = synth.make_qkv_device(cfg, dev)
     dt = hb._DT[q.dtype]
     qkv = hb.alloc_qkv(cfg.B, cfg.Hq, cfg.Hkv, cfg.N, cfg.d, dt, dev, qmean=qmean)
@@ -179,13 +180,17 @@ def time_workload(hb, cfg, dev, steps, warmup, flush_l2, s=None, inv_s=None, qme
     status = torch.zeros(1, dtype=torch.int32, device=dev)
 
     def step(split):
-        hb.quantize_qkv(q, k, v, s, inv_s, out=qkv, d_status=status, qmean=qmean)
+        hb.quantize_qkv(None if fused_q else q, k, v, s, inv_s, out=qkv, d_status=status, qmean=qmean, Hq=cfg.Hq)
         mid = None
         if split:
             mid = torch.cuda.Event(enable_timing=True)
             mid.record()
-        hb.attention_fwd(qkv, cfg.causal, Bc=cfg.Bc, out_dtype=hb.F32, out=out, d_status=status,
-                         p_dtype=hb.F32 if p_f32 else hb.F16, qmean=qmean)
+        if fused_q:
+            hb.attention_fwd_qraw(q, s, qkv, cfg.causal, out_dtype=hb.F32, out=out, d_status=status,
+                                  p_dtype=hb.F32 if p_f32 else hb.F16)
+        else:
+            hb.attention_fwd(qkv, cfg.causal, Bc=cfg.Bc, out_dtype=hb.F32, out=out, d_status=status,
+                             p_dtype=hb.F32 if p_f32 else hb.F16, qmean=qmean)
         return mid
 
     for _ in range(warmup):
@@ -572,6 +577,8 @@ def main():
                    ("C2 Bc=128", synth.config("C2", Bc=128), {}),
                    ("C2 Q-Mean", synth.config("C2"), {"qmean": True}),
                    ("C2 FP32-P variant", synth.config("C2"), {"p_f32": True}),
+                   ("C2 Q quantized inside the attention kernel", synth.config("C2"), {"fused_q": True}),
+                   ("C2@8192 Q quantized inside the attention kernel", synth.config("C2", N=8192), {"fused_q": True}),
                    ("C3", synth.config("C3"), {}), ("C4", synth.config("C4"), {})]
         for n_ in (1024, 2048, 4096, 8192, 16384, 32768):
             entries.append((f"C5@{n_} causal", synth.config("C5", N=n_), {}))

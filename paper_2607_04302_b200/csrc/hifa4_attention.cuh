@@ -65,69 +65,6 @@ struct Cfg {
 
 __device__ __forceinline__ float f16_round(float x) { return __half2float(__float2half_rn(x)); }
 
-// Algorithm 1 line 1 inside the attention kernel: one thread turns the 64 channels of one raw query row that TMA
-// left in shared memory (a 128-byte row of a swizzled 64-channel sub-tile; `row_addr` its start, `sw` = row % 8 the
-// swizzle key) into the BF16 image of HIF4(round_in(q * s)), in place.  scale: the 64 Smooth-QK factors of these
-// channels or null.  The arithmetic is that of the stand-alone quantizer (hif4_group / hif4_unit), with the whole
-// group in one thread instead of an 8-lane team.
-template <typename T>
-__device__ __forceinline__ void quantize_q_row_inplace(uint32_t row_addr, int sw, const float* __restrict__ scale)
-{
-    uint32_t xw[32];
-#pragma unroll
-    for (int c = 0; c < 8; ++c)
-        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                     : "=r"(xw[4 * c]), "=r"(xw[4 * c + 1]), "=r"(xw[4 * c + 2]), "=r"(xw[4 * c + 3])
-                     : "r"(row_addr + (uint32_t)((c ^ sw) << 4)));
-    float A = 0.f;
-#pragma unroll
-    for (int c = 0; c < 8; ++c) {
-        float sv[8];
-        if (scale) {
-            const float4 s0 = __ldg(reinterpret_cast<const float4*>(scale) + 2 * c);
-            const float4 s1 = __ldg(reinterpret_cast<const float4*>(scale) + 2 * c + 1);
-            sv[0] = s0.x; sv[1] = s0.y; sv[2] = s0.z; sv[3] = s0.w;
-            sv[4] = s1.x; sv[5] = s1.y; sv[6] = s1.z; sv[7] = s1.w;
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            float lo, hi;
-            Pair16<T>::unpack(xw[4 * c + i], lo, hi);
-            if (scale) {                                   // FP32 product, rounded once to the activation dtype
-                float a, b;
-                unpack2(mul2(pack2(lo, hi), pack2(sv[2 * i], sv[2 * i + 1])), a, b);
-                xw[4 * c + i] = Pair16<T>::round_pack(a, b);
-                Pair16<T>::unpack(xw[4 * c + i], lo, hi);
-            }
-            A = max3(A, fabsf(lo), fabsf(hi));
-        }
-    }
-    const Hif4Group g = hif4_group(A);                     // A = 0: code 0 and an all-zero group
-    const bool sat = A > g.top;                            // only above the E6M2 range
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-        float x[8], y[8];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) Pair16<T>::unpack(xw[4 * u + i], x[2 * i], x[2 * i + 1]);
-        if (sat) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) x[i] = fminf(fmaxf(x[i], -g.top), g.top);
-        }
-        const float a0 = fmaxf(max3(fabsf(x[0]), fabsf(x[1]), fabsf(x[2])), fabsf(x[3]));
-        const float a1 = fmaxf(max3(fabsf(x[4]), fabsf(x[5]), fabsf(x[6])), fabsf(x[7]));
-        uint32_t w[4];
-        int a, k0, k1;
-        hif4_unit(x, a0, a1, g, w, y, a, k0, k1);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) xw[4 * u + i] = w[i];
-    }
-#pragma unroll
-    for (int c = 0; c < 8; ++c)
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                     ::"r"(row_addr + (uint32_t)((c ^ sw) << 4)), "r"(xw[4 * c]), "r"(xw[4 * c + 1]), "r"(xw[4 * c + 2]),
-                       "r"(xw[4 * c + 3]) : "memory");
-}
-
 // exp2 of two values, each result rounded to FP16 (one packed conversion) and widened back.
 __device__ __forceinline__ void exp2_f16_pair(float t0, float t1, float& e0, float& e1)
 {

@@ -54,8 +54,9 @@ struct WS64 {
     static constexpr int K_OFF = Q_OFF + Q_BYTES;
     static constexpr int V_OFF = K_OFF + STAGES * K_STAGE;
     static constexpr int MISC_OFF = V_OFF + STAGES * V_STAGE;
-    static constexpr int KSUM_OFF = MISC_OFF + 256;         // Q-Mean: channel sums of the tile's 64 keys, two stages
-    static constexpr int MX_OFF = KSUM_OFF + STAGES * 256;  // running maxima handed from tile j to tile j+1: [2][128] floats
+    static constexpr int KSUM_SLOTS = 4;                    // Q-Mean: channel sums of a tile's 64 keys; slot = tile % 4
+    static constexpr int KSUM_OFF = MISC_OFF + 256;
+    static constexpr int MX_OFF = KSUM_OFF + KSUM_SLOTS * 256;  // running maxima handed from tile j to tile j+1: [2][128] floats
     static constexpr int SMEM_BYTES = MX_OFF + 2 * 512 + 1024;
     static constexpr int O_COLS = D + 16;
     static constexpr bool Q_IN_TMEM = (D == 256);
@@ -69,11 +70,11 @@ namespace ws64 {
 // Index s = tile % 2 everywhere.  QKGO[s]: K stage s has landed and S is free (4 arrivals + 1 + bytes); PVGO[s]:
 // V^T stage s has landed, the image of P-hat is stored and [O | l] rescaled (4 arrivals + 1 + bytes); KE / VE:
 // stage free (MMA commit); SF[s]: S complete; PV[s]: P V complete; MR[s]: running maxima after the tile
-// published (4 arrivals); KSF[s]: Q-Mean key sums landed; QT: Q-hat image copied to tensor memory.
+// published (4 arrivals); KSF[tile % 4]: Q-Mean key sums landed (a barrier per slot); QT: Q-hat image copied to tensor memory.
 // Two barriers per kind because each group of softmax warps sees every second tile only: a parity wait
 // must observe every phase of its barrier.
 enum { BAR_Q = 0, BAR_QKGO = 1, BAR_KE = 3, BAR_PVGO = 5, BAR_VE = 7, BAR_SF = 9, BAR_PV = 11, BAR_KSF = 13,
-       BAR_MR = 15, BAR_QT = 17, N_BARS = 18 };
+       BAR_MR = 17, BAR_QT = 19, N_BARS = 20 };
 constexpr uint32_t WAIT_POLLS = 1u << 20;
 }  // namespace ws64
 
@@ -149,17 +150,21 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
 #pragma unroll
         for (int s = 0; s < QSUB; ++s)
             tma_load_3d(k_s + st * K_STAGE + s * K_SUB, &tmap_k, bar(BAR_QKGO + st), 64 * s, jt * BC, bh_kv);
+        if (QM) {
+            // Q-Mean: the 64 channel sums of this tile's keys travel with the K tile, two tiles ahead of their use
+            // right after S is pulled (with the V^T tile they arrived ~2000 clk after the softmax warps wanted
+            // them).  Four slots with a barrier each: slot jt % 4 held the sums of tile jt-4, whose readers arrived
+            // on the barrier that released S(jt-3) only after reading them, and this load follows S(jt-2).  (Two
+            // barriers would not do: the sums of tile jt+2 can land before a late reader has looked for those of
+            // tile jt, and a parity wait that is two phases behind never returns.)
+            mbar_expect_tx(bar(BAR_KSF + (jt & 3)), 256);
+            bulk_load(smem_base + C::KSUM_OFF + (jt & 3) * 256, args.k_sum + (size_t)bh_kv * N + jt * BC, 256, bar(BAR_KSF + (jt & 3)));
+        }
     };
     auto load_v = [&](int jt) {                               // V^T tile jt into stage jt % 2
         const int st = jt & 1;
         mbar_expect_tx(bar(BAR_PVGO + st), D * 128);
         tma_load_3d(v_s + st * V_STAGE, &tmap_v, bar(BAR_PVGO + st), jt * BC, 0, bh_kv);
-        if (QM) {
-            // Q-Mean: the 64 channel sums of this tile's keys; their stage is free with the V stage
-            // (P V of tile jt-2 complete means every softmax warp is past tile jt-2)
-            mbar_expect_tx(bar(BAR_KSF + st), 256);
-            bulk_load(smem_base + C::KSUM_OFF + st * 256, args.k_sum + (size_t)bh_kv * N + jt * BC, 256, bar(BAR_KSF + st));
-        }
     };
 
     if (warp == W_QK && lane == 0) {
@@ -174,7 +179,7 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             mbar_init(bar(BAR_QKGO + s), 5); mbar_init(bar(BAR_KE + s), 1);
             mbar_init(bar(BAR_PVGO + s), 5); mbar_init(bar(BAR_VE + s), 1);
             mbar_init(bar(BAR_SF + s), 1); mbar_init(bar(BAR_PV + s), 1);
-            mbar_init(bar(BAR_KSF + s), 1); mbar_init(bar(BAR_MR + s), 4);
+            mbar_init(bar(BAR_KSF + s), 1); mbar_init(bar(BAR_KSF + 2 + s), 1); mbar_init(bar(BAR_MR + s), 4);
         }
         mbar_init(bar(BAR_QT), NSW);
         fence_barrier_init();
@@ -317,8 +322,8 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             if (wait64(bar(BAR_Q), 0, abort_flag)) {
                 const uint32_t row_addr = q_s + (uint32_t)kq * 16384u + (uint32_t)r_loc * 128u;
                 const float* sc = args.q_scale ? args.q_scale + (size_t)g * D + kq * 64 : nullptr;
-                if (args.in_dtype == HIFA4_F16) quantize_q_row_inplace<__half>(row_addr, r_loc & 7, sc);
-                else quantize_q_row_inplace<__nv_bfloat16>(row_addr, r_loc & 7, sc);
+                if (args.in_dtype == HIFA4_F16) hif4_quantize_row64_inplace<__half>(row_addr, r_loc & 7, sc);
+                else hif4_quantize_row64_inplace<__nv_bfloat16>(row_addr, r_loc & 7, sc);
             } else { fail(13); ok = false; }
             fence_proxy_async_smem();                          // generic-proxy writes, read by the MMA
             __syncwarp();
@@ -343,21 +348,22 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             }
             tc_fence_before();                                 // S(jt) is in registers: S(jt+1) may overwrite it
             __syncwarp();
-            if (jt + 1 < n_tiles) arrive_lane0(bar(BAR_QKGO + (st ^ 1)), lane);
+            if (!QM && jt + 1 < n_tiles) arrive_lane0(bar(BAR_QKGO + (st ^ 1)), lane);
 
             if (QM) {                                          // Q-Mean correction (line 6): + mu_i * sum_c k~_jc
-                if (!wait64(bar(BAR_KSF + st), ph, abort_flag)) { fail(15); ok = false; break; }
-                const uint32_t ks_s = smem_base + C::KSUM_OFF + st * 256;
+                if (!wait64(bar(BAR_KSF + (jt & 3)), (uint32_t)(jt >> 2) & 1u, abort_flag)) { fail(15); ok = false; break; }
+                const uint32_t ks_s = smem_base + C::KSUM_OFF + (jt & 3) * 256;
+                const uint64_t mu2 = pack2(mu_row, mu_row);
 #pragma unroll
                 for (int i = 0; i < BC / 4; ++i) {
                     float4 ks;
                     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
                                  : "=f"(ks.x), "=f"(ks.y), "=f"(ks.z), "=f"(ks.w) : "r"(ks_s + 16 * i));
-                    p[4 * i] = fmaf(mu_row, ks.x, p[4 * i]);
-                    p[4 * i + 1] = fmaf(mu_row, ks.y, p[4 * i + 1]);
-                    p[4 * i + 2] = fmaf(mu_row, ks.z, p[4 * i + 2]);
-                    p[4 * i + 3] = fmaf(mu_row, ks.w, p[4 * i + 3]);
+                    unpack2(fma2(mu2, pack2(ks.x, ks.y), pack2(p[4 * i], p[4 * i + 1])), p[4 * i], p[4 * i + 1]);
+                    unpack2(fma2(mu2, pack2(ks.z, ks.w), pack2(p[4 * i + 2], p[4 * i + 3])), p[4 * i + 2], p[4 * i + 3]);
                 }
+                __syncwarp();                                  // the slot has been read: only now may S(jt+1) go
+                if (jt + 1 < n_tiles) arrive_lane0(bar(BAR_QKGO + (st ^ 1)), lane);
             }
             if ((args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N)) {   // masked scores become -inf: exp gives exact zeros
 #pragma unroll

@@ -150,4 +150,102 @@ __device__ __forceinline__ void hif4_unit(const float (&x)[8], float a0, float a
     }
 }
 
+// Packed sign-magnitude nibbles of one level-2 unit from the biased quotients y of hif4_unit: element i in nibble i.
+// The low byte of bits(y) is the signed code m (the magic constant's low byte is 0): the bytes are gathered and
+// turned into sign-magnitude nibbles with byte-parallel arithmetic.
+__device__ __forceinline__ uint32_t hif4_unit_nibbles(const float (&y)[8])
+{
+    uint32_t xw[2];                                               // per subgroup: nibbles n0 | n1 << 4 in byte 0, n2 | n3 << 4 in byte 2
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t b01 = __byte_perm(__float_as_uint(y[4 * h]), __float_as_uint(y[4 * h + 1]), 0x0040);
+        const uint32_t b23 = __byte_perm(__float_as_uint(y[4 * h + 2]), __float_as_uint(y[4 * h + 3]), 0x0040);
+        const uint32_t bb = __byte_perm(b01, b23, 0x5410);                     // m0, m1, m2, m3 as signed bytes
+        const uint32_t sg = bb & 0x80808080u;                                  // sign bits
+        const uint32_t ng = sg >> 7;                                           // 1 in every negative byte
+        const uint32_t ab = (bb ^ (ng * 0xFFu)) + ng;                          // |m| per byte (no carry between bytes: |m| <= 7)
+        const uint32_t nb = ab | (sg >> 4);                                    // sign to bit 3 of the byte
+        xw[h] = nb | (nb >> 4);
+    }
+    return __byte_perm(xw[0], xw[1], 0x6420);
+}
+// The unit's share of the group's metadata word: level-2 bit at 8 + j, the two level-3 bits at 16 + 2 j (j = unit
+// index in the group); the scale code (bits 0..7) is added once per group.
+__device__ __forceinline__ uint32_t hif4_unit_meta(int j, int a, int k0, int k1)
+{
+    return ((uint32_t)a << (8 + j)) | ((uint32_t)((k0 - a) | ((k1 - a) << 1)) << (16 + 2 * j));
+}
+
+// One thread quantizes one whole 64-element group (Algorithm 1 lines 1 and 3) held in registers as 32 words of
+// 16-bit pairs (element 2i in the low half of word i): the words are replaced by the BF16 image of
+// HIF4(round_in(x * s)).  scale: the 64 Smooth-QK factors of these elements or null.  Same arithmetic as the 8-lane
+// team of the stand-alone quantizer (hif4_group / hif4_unit), with the group constants formed once and no shuffles;
+// the packed codes are not formed (the caller consumes the image at once).
+template <typename T>
+__device__ __forceinline__ void hif4_quantize64_regs(uint32_t (&xw)[32], const float* __restrict__ scale)
+{
+    float Ap[4] = {0.f, 0.f, 0.f, 0.f};                    // four independent maximum chains
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        float sv[8];
+        if (scale) {
+            const float4 s0 = __ldg(reinterpret_cast<const float4*>(scale) + 2 * c);
+            const float4 s1 = __ldg(reinterpret_cast<const float4*>(scale) + 2 * c + 1);
+            sv[0] = s0.x; sv[1] = s0.y; sv[2] = s0.z; sv[3] = s0.w;
+            sv[4] = s1.x; sv[5] = s1.y; sv[6] = s1.z; sv[7] = s1.w;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            float lo, hi;
+            Pair16<T>::unpack(xw[4 * c + i], lo, hi);
+            if (scale) {                                   // FP32 product, rounded once to the activation dtype
+                float a, b;
+                unpack2(mul2(pack2(lo, hi), pack2(sv[2 * i], sv[2 * i + 1])), a, b);
+                xw[4 * c + i] = Pair16<T>::round_pack(a, b);
+                Pair16<T>::unpack(xw[4 * c + i], lo, hi);
+            }
+            Ap[i] = max3(Ap[i], fabsf(lo), fabsf(hi));
+        }
+    }
+    const float A = fmaxf(max3(Ap[0], Ap[1], Ap[2]), Ap[3]);
+    const Hif4Group g = hif4_group(A);                     // A = 0: code 0 and an all-zero group
+    const bool sat = A > g.top;                            // only above the E6M2 range
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        float x[8], y[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) Pair16<T>::unpack(xw[4 * u + i], x[2 * i], x[2 * i + 1]);
+        if (sat) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[i] = fminf(fmaxf(x[i], -g.top), g.top);
+        }
+        const float a0 = fmaxf(max3(fabsf(x[0]), fabsf(x[1]), fabsf(x[2])), fabsf(x[3]));
+        const float a1 = fmaxf(max3(fabsf(x[4]), fabsf(x[5]), fabsf(x[6])), fabsf(x[7]));
+        uint32_t w[4];
+        int a, k0, k1;
+        hif4_unit(x, a0, a1, g, w, y, a, k0, k1);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) xw[4 * u + i] = w[i];
+    }
+}
+
+// The same for a group that sits in shared memory as a 128-byte row of a 64-column tile with the 128-byte swizzle
+// TMA applies (`row_addr` the row's start, `sw` = row % 8 the swizzle key): quantized in place.
+template <typename T>
+__device__ __forceinline__ void hif4_quantize_row64_inplace(uint32_t row_addr, int sw, const float* __restrict__ scale)
+{
+    uint32_t xw[32];
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(xw[4 * c]), "=r"(xw[4 * c + 1]), "=r"(xw[4 * c + 2]), "=r"(xw[4 * c + 3])
+                     : "r"(row_addr + (uint32_t)((c ^ sw) << 4)));
+    hif4_quantize64_regs<T>(xw, scale);
+#pragma unroll
+    for (int c = 0; c < 8; ++c)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                     ::"r"(row_addr + (uint32_t)((c ^ sw) << 4)), "r"(xw[4 * c]), "r"(xw[4 * c + 1]), "r"(xw[4 * c + 2]),
+                       "r"(xw[4 * c + 3]) : "memory");
+}
+
 }  // namespace hifa4

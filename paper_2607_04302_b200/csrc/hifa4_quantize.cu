@@ -34,23 +34,9 @@ __device__ __forceinline__ uint32_t quantize8(float (&x)[8], int j, uint32_t (&w
     float y[8];
     int a, k0, k1;
     hif4_unit(x, a0, a1, g, w, y, a, k0, k1);
-    uint32_t part = ((uint32_t)a << (8 + j)) | ((uint32_t)((k0 - a) | ((k1 - a) << 1)) << (16 + 2 * j));
+    uint32_t part = hif4_unit_meta(j, a, k0, k1);
     if (j == 0) part |= (uint32_t)g.code;
-    uint32_t xw[2];                                               // per subgroup: nibbles n0 | n1 << 4 in byte 0, n2 | n3 << 4 in byte 2
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        // The low byte of bits(y) is the signed code m (the magic constant's low byte is 0): gather the
-        // four bytes and turn them into sign-magnitude nibbles with byte-parallel arithmetic.
-        const uint32_t b01 = __byte_perm(__float_as_uint(y[4 * h]), __float_as_uint(y[4 * h + 1]), 0x0040);
-        const uint32_t b23 = __byte_perm(__float_as_uint(y[4 * h + 2]), __float_as_uint(y[4 * h + 3]), 0x0040);
-        const uint32_t bb = __byte_perm(b01, b23, 0x5410);                     // m0, m1, m2, m3 as signed bytes
-        const uint32_t sg = bb & 0x80808080u;                                  // sign bits
-        const uint32_t ng = sg >> 7;                                           // 1 in every negative byte
-        const uint32_t ab = (bb ^ (ng * 0xFFu)) + ng;                          // |m| per byte (no carry between bytes: |m| <= 7)
-        const uint32_t nb = ab | (sg >> 4);                                    // sign to bit 3 of the byte
-        xw[h] = nb | (nb >> 4);
-    }
-    const uint32_t nib = __byte_perm(xw[0], xw[1], 0x6420);
+    const uint32_t nib = hif4_unit_nibbles(y);
     part |= __shfl_xor_sync(0xffffffffu, part, 1);
     part |= __shfl_xor_sync(0xffffffffu, part, 2);
     part |= __shfl_xor_sync(0xffffffffu, part, 4);
