@@ -358,3 +358,66 @@ def test_in_kernel_query_quantization_full_size_and_refusals(hb, par):
     q6, k6, v6 = (t.to(DEV) for t in synth.make_qkv(c64))
     with pytest.raises(hb.Hifa4Error):
         hb.attention_fwd_qraw(q6, None, hb.quantize_qkv(None, k6, v6, Hq=1), True)
+
+
+def test_calls_are_capturable_in_a_cuda_graph_and_replay_bit_identically(hb, par):
+    """The entry points allocate nothing, synchronise nothing and only enqueue work on the caller's stream, so a
+    quantize + attention pair (the grid with programmatic stream serialization included) and the raw entry point
+    can be captured in a CUDA graph; replays write the same bits as the eager calls, also after the inputs changed
+    in place."""
+    cfg = synth.config("C2", B=1, Hq=8, Hkv=2, N=1024)
+    q, k, v = (t.to(DEV) for t in synth.make_qkv(cfg))
+    s, inv_s = par.calibrate(cfg, DEV)
+    qkv = hb.quantize_qkv(q, k, v, s, inv_s)
+    want = hb.attention_fwd(qkv, True)                                   # eager: also opts the kernels in
+    want_raw = hb.attention_fwd_raw(q, k, v, s, inv_s, True)
+    assert torch.equal(want, want_raw)
+    out = torch.zeros_like(want)
+    out_raw = torch.zeros_like(want)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    ws = torch.empty(hb.attention_raw_workspace_bytes(cfg.B, cfg.Hq, cfg.Hkv, cfg.N, cfg.d, qkv.in_dtype, True, 64),
+                     dtype=torch.uint8, device=DEV)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=torch.cuda.Stream(device=DEV)):
+        hb.quantize_qkv(q, k, v, s, inv_s, out=qkv, d_status=status)
+        hb.attention_fwd(qkv, True, out=out, d_status=status)
+        hb.attention_fwd_raw(q, k, v, s, inv_s, True, out=out_raw, workspace=ws, d_status=status)
+    g.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(out, want) and torch.equal(out_raw, want)
+    q2 = q.flip(2).contiguous()
+    want2 = hb.attention_fwd(hb.quantize_qkv(q2, k, v, s, inv_s), True)
+    q.copy_(q2)                                                          # same buffers, new contents
+    g.replay()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(out, want2) and torch.equal(out_raw, want2)
+    assert not torch.equal(want, want2)
+
+
+def test_concurrent_host_threads_on_their_own_streams(hb, par):
+    """Two host threads call the library at the same time, each on its own stream and buffers (the per-device
+    shared-memory opt-in and the tensor-map encoder look-up are guarded): both get the serial result."""
+    import threading
+    cfgs = [synth.config("C2", B=1, Hq=4, Hkv=2, N=512, seed=11), synth.config("C3", B=1, Hq=4, Hkv=1, N=768, seed=12)]
+    data = [tuple(t.to(DEV) for t in synth.make_qkv(c)) for c in cfgs]
+    want = [hb.attention_fwd(hb.quantize_qkv(*d), c.causal) for c, d in zip(cfgs, data)]
+    torch.cuda.synchronize()
+    got, errs = [None, None], []
+
+    def work(i):
+        try:
+            with torch.cuda.stream(torch.cuda.Stream(device=DEV)):
+                for _ in range(20):
+                    got[i] = hb.attention_fwd_raw(*data[i], None, None, cfgs[i].causal)
+                torch.cuda.current_stream().synchronize()
+        except Exception as e:                                           # surfaced below
+            errs.append(e)
+
+    ts = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+    for t in ts:
+        t.start()
+    for t in ts:
+        t.join()
+    assert not errs, errs
+    assert torch.equal(got[0], want[0]) and torch.equal(got[1], want[1])
