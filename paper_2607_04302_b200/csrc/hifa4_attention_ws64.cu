@@ -14,9 +14,9 @@
 // stage two tiles ahead; the next MMA of the same kind cannot start earlier anyway (the next S needs the
 // softmax warps to have pulled this S, the next P V needs the P-hat that follows this P V).
 // Each MMA waits on ONE barrier: the barrier that releases S of a tile collects the bytes of the K tile
-// (TMA transaction count) and the eight "S is in registers" arrivals of the softmax warps, the one that
-// releases P V collects the bytes of the V^T tile and the eight "P-hat stored, history rescaled"
-// arrivals.  The two issuers run independently: a late P V never delays the next S (device timestamps
+// (TMA transaction count) and the four "S is in registers" arrivals of the group that owns the previous tile,
+// the one that releases P V collects the bytes of the V^T tile and the four "P-hat stored, history rescaled"
+// arrivals of the tile's owners.  The two issuers run independently: a late P V never delays the next S (device timestamps
 // of a single in-order issuer showed S(j+1) issued 1500 clk after it could have been).
 // S has a single buffer that is released early: the softmax warps pull S(j) into registers and
 // signal it free, and S(j+1) runs on the tensor pipe while they work on tile j; the BF16 image of P-hat
@@ -29,12 +29,14 @@
 //   d = 128: 256 tensor-memory columns: [O | l] 0..143 (one N = 144 MMA), S 144..207, P-hat
 //            208..239; Q-hat stays in shared memory (SS-form Q K^T).  101 KB of shared memory, so two
 //            CTAs share an SM and fill each other's synchronisation gaps.
-// Polls for S(j+1) and PV(j-1) are issued early with test_wait (try_wait blocks while the phase is
-// incomplete); the blocking wait is the fall-back.  Epilogue: O / l by reciprocal plus one correction
+// Every wait polls with test_wait (a thread suspended in try_wait was seen to notice a completed phase about
+// 1000 clk late).  Epilogue: O / l by reciprocal plus one correction
 // step, FP32 output through a per-warp 32 x 32 shared-memory transpose (the K stages are idle by then).
 // The grid is launched with programmatic stream serialization: everything before griddepcontrol.wait
 // (barrier set-up, tensor-memory allocation) may overlap the tail of the preceding kernel.
-// Template flags: P-hat dump, FP32-P variant, Q-Mean (key sums staged in shared memory by the producer).
+// Template flags: P-hat dump, FP32-P variant, Q-Mean (the K thread stages each tile's key sums in shared memory,
+// two tiles ahead), self-test (one wait made to run out), raw Q (Q smoothed and quantized in shared memory by
+// the softmax threads before the first S).
 // Every wait is bounded (see hifa4_attention_ws.cu for the failure protocol).
 #include "hifa4_attention.cuh"
 
