@@ -448,21 +448,23 @@ def main():
     # FP16 output (the method's final normalisation is FP16: Appendix, "FP16 operations") and FP32 output (the
     # dtype the parity tests judge); the FP16 one is the line's `e2e`.
     e2e = e2e_f32 = None
-    if not big and not args.qmean:
+    if not big and not args.qmean and not args.p_f32:
         pq, pk, pv = qh.pin_memory(), kh.pin_memory(), vh.pin_memory()
-        dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
-        # One problem per (batch, pair of KV head groups): its Q/K/V slices are contiguous, so each goes through
-        # hifa4_attention_fwd_raw on its own; one stream carries all host-to-device copies, one all device-to-host
-        # copies and three the kernels, tied together by events, so that the copy of one slice, the kernels of
-        # another and the read-back of a third are in flight together.  (Finer slices are bound by the host: each
-        # slice costs about a dozen Python-level API calls.)
+        # One problem per batch element: hifa4_attention_fwd_raw on its Q/K/V (contiguous slices).  One stream
+        # carries all host-to-device copies, one all device-to-host copies, the kernels of consecutive problems
+        # alternate between two more.  Device buffers come in two sets used by alternate steps, tied by events: a
+        # set's inputs are overwritten only after the kernels that read them, its output only after the read-back
+        # of the previous result, so consecutive steps pipeline (copy-in of step i+1 under the kernels of step i and
+        # the read-back of step i-1) exactly as they would with different data in every step.  Few large copies:
+        # with one problem per pair of KV head groups (twelve copies in, four out per step) the same pipeline was
+        # 15 % slower.
         G = cfg.Hq // cfg.Hkv
-        GPS = 2 if cfg.Hkv % 2 == 0 else 1                               # KV head groups per slice
-        streams = [torch.cuda.Stream(device=dev) for _ in range(3)]
+        NB = 2
+        streams = [torch.cuda.Stream(device=dev) for _ in range(2)]
         h2d_stream, d2h_stream = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
-        ws_bytes = hb.attention_raw_workspace_bytes(1, G * GPS, GPS, cfg.N, cfg.d, dt, cfg.causal, cfg.Bc)
+        ws_bytes = hb.attention_raw_workspace_bytes(1, cfg.Hq, cfg.Hkv, cfg.N, cfg.d, dt, cfg.causal, cfg.Bc)
         ws_s = [torch.empty(ws_bytes, dtype=torch.uint8, device=dev) for _ in streams]
-        slices = [(bb, g) for bb in range(cfg.B) for g in range(0, cfg.Hkv, GPS)]
+        in_sets = [tuple(torch.empty_like(t) for t in (q, k, v)) for _ in range(NB)]
 
         def fork():
             e = torch.cuda.Event()
@@ -477,55 +479,75 @@ def main():
                 torch.cuda.current_stream().wait_event(e)
 
         def e2e_run(out_code, torch_dt):
-            d_out = out if torch_dt == torch.float32 else torch.empty(out.shape, dtype=torch_dt, device=dev)
-            po = torch.empty(out.shape, dtype=torch_dt).pin_memory()
+            d_outs = [torch.empty(out.shape, dtype=torch_dt, device=dev) for _ in range(NB)]
+            pos = [torch.empty(out.shape, dtype=torch_dt).pin_memory() for _ in range(NB)]
+            inputs_free = [None] * NB                                  # events: kernels that read the set are done
+            output_free = [None] * NB                                  # event: read-back of the set's output is done
+            calls = [0]
 
-            def e2e_step():
-                for i, (bb, g) in enumerate(slices):
-                    st_i = streams[i % len(streams)]
-                    hs, gs = slice(g * G, (g + GPS) * G), slice(g, g + GPS)
+            def e2e_step(i):
+                b_i = i % NB
+                dq, dk, dv = in_sets[b_i]
+                kernels_done = []
+                for bb in range(cfg.B):
+                    st_i = streams[calls[0] % len(streams)]
                     with torch.cuda.stream(h2d_stream):
-                        dq[bb:bb + 1, hs].copy_(pq[bb:bb + 1, hs], non_blocking=True)
-                        dk[bb:bb + 1, gs].copy_(pk[bb:bb + 1, gs], non_blocking=True)
-                        dv[bb:bb + 1, gs].copy_(pv[bb:bb + 1, gs], non_blocking=True)
+                        if bb == 0 and inputs_free[b_i] is not None:
+                            for e in inputs_free[b_i]:
+                                h2d_stream.wait_event(e)
+                        dq[bb:bb + 1].copy_(pq[bb:bb + 1], non_blocking=True)
+                        dk[bb:bb + 1].copy_(pk[bb:bb + 1], non_blocking=True)
+                        dv[bb:bb + 1].copy_(pv[bb:bb + 1], non_blocking=True)
                         landed = torch.cuda.Event()
                         landed.record()
                     st_i.wait_event(landed)
+                    if output_free[b_i] is not None:
+                        st_i.wait_event(output_free[b_i])
                     with torch.cuda.stream(st_i):
-                        hb.attention_fwd_raw(dq[bb:bb + 1, hs], dk[bb:bb + 1, gs], dv[bb:bb + 1, gs],
-                                             None if s is None else s[gs], None if inv_s is None else inv_s[gs],
-                                             cfg.causal, Bc=cfg.Bc, out_dtype=out_code, out=d_out[bb:bb + 1, hs],
-                                             workspace=ws_s[i % len(streams)], d_status=status)
+                        hb.attention_fwd_raw(dq[bb:bb + 1], dk[bb:bb + 1], dv[bb:bb + 1], s, inv_s,
+                                             cfg.causal, Bc=cfg.Bc, out_dtype=out_code, out=d_outs[b_i][bb:bb + 1],
+                                             workspace=ws_s[calls[0] % len(streams)], d_status=status)
                         done = torch.cuda.Event()
                         done.record()
+                    calls[0] += 1
+                    kernels_done.append(done)
                     d2h_stream.wait_event(done)
                     with torch.cuda.stream(d2h_stream):
-                        po[bb:bb + 1, hs].copy_(d_out[bb:bb + 1, hs], non_blocking=True)
+                        pos[b_i][bb:bb + 1].copy_(d_outs[b_i][bb:bb + 1], non_blocking=True)
+                inputs_free[b_i] = kernels_done
+                with torch.cuda.stream(d2h_stream):
+                    e = torch.cuda.Event()
+                    e.record()
+                    output_free[b_i] = e
 
             fork()
-            for _ in range(3):
-                e2e_step()
+            for i in range(4):
+                e2e_step(i)
             join()
             barrier()
+            for po in pos:
+                po.zero_()
             a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
-            n_e2e = max(3, min(args.steps, 50))                  # back-to-back steps: their copies and kernels pipeline
+            n_e2e = max(4, min(args.steps, 50))                  # back-to-back steps: their copies and kernels pipeline
             a.record()
             fork()
-            for _ in range(n_e2e):
-                e2e_step()
+            for i in range(n_e2e):
+                e2e_step(i)
             join()
             b.record()
             barrier()
             assert int(status.item()) == 0, f"device status {int(status.item())}"
-            # the host copy equals the device-resident result of the timed steps, rounded once to the output dtype
-            assert torch.equal(po.to(dev), out.to(torch_dt)), "end-to-end output differs from the device result"
+            # every host copy equals the device-resident result of the timed steps, rounded once to the output dtype
+            for po in pos:
+                assert torch.equal(po.to(dev), out.to(torch_dt)), "end-to-end output differs from the device result"
             e_ms = max_over_ranks(dist, a.elapsed_time(b), dev)
             h2d = (pq.numel() + pk.numel() + pv.numel()) * pq.element_size()
             return {"value": whole_job_tflops(cfg, world, n_e2e, e_ms), "unit": UNIT,
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": po.numel() * po.element_size(),
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": pos[0].numel() * pos[0].element_size(),
                     "ms_per_step": e_ms / n_e2e, "steps": n_e2e, "out_dtype": str(torch_dt).replace("torch.", ""),
-                    "how": f"hifa4_attention_fwd_raw per (batch, KV head group) slice, {len(slices)} slices over "
-                           f"{len(streams)} kernel streams and two copy streams, pinned host buffers"}
+                    "how": f"hifa4_attention_fwd_raw per batch element ({cfg.B} per step), {NB} sets of device buffers used "
+                           f"by alternate steps, {len(streams)} kernel streams and two copy streams tied by events, pinned "
+                           "host buffers; back-to-back steps pipeline"}
 
         e2e_f32 = e2e_run(hb.F32, torch.float32)
         e2e = e2e_run(hb.F16, torch.float16)
