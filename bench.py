@@ -139,8 +139,9 @@ def whole_job_tflops(cfg, world: int, steps: int, total_ms: float) -> float:
 
 
 def measure_gemm_peaks(dev):
-    """Dense GEMM throughput measured in this run (8192^3, best of 5): BF16 through torch.matmul, FP8 (e4m3)
-    through torch._scaled_mm; FP4 only if the installed torch exposes a dense FP4 matmul (it does not: null)."""
+    """Dense GEMM throughput measured in this run (8192^3, best of 5): BF16 through torch.matmul, FP8 (e4m3) and
+    FP4 (e2m1 with one e4m3 scale per 16 elements, the block-scaled 4-bit format the tensor cores take) through
+    torch._scaled_mm; each is null where the installed torch does not expose it."""
     res = {"bf16_tflops": None, "fp8_tflops": None, "fp4_tflops": None}
     n = 8192
     try:
@@ -166,6 +167,14 @@ def measure_gemm_peaks(dev):
         res["fp8_tflops"] = best(lambda: torch._scaled_mm(a8, b8, scale_a=one, scale_b=one, out_dtype=torch.bfloat16))
     except Exception as e:                                             # context only: never fail the bench on it
         res["error"] = str(e)[:160]
+    try:
+        # random 4-bit codes, all block scales 1.0 in the 128 x 4 tiled layout the block-scaled GEMM reads
+        a4 = torch.randint(0, 256, (n, n // 2), dtype=torch.uint8, device=dev).view(torch.float4_e2m1fn_x2)
+        b4 = torch.randint(0, 256, (n, n // 2), dtype=torch.uint8, device=dev).view(torch.float4_e2m1fn_x2)
+        sc = torch.ones((n * (n // 16),), device=dev, dtype=torch.float32).to(torch.float8_e4m3fn)
+        res["fp4_tflops"] = best(lambda: torch._scaled_mm(a4, b4.t(), scale_a=sc, scale_b=sc, out_dtype=torch.bfloat16))
+    except Exception as e:
+        res["fp4_error"] = str(e)[:160]
     return res
 
 
@@ -640,6 +649,8 @@ def main():
             frac_measured["fp4_as_4x_bf16_this_run"] = achieved / (4 * gemm["bf16_tflops"])
         if gemm.get("fp8_tflops"):
             frac_measured["fp8_this_run"] = achieved / gemm["fp8_tflops"]
+        if gemm.get("fp4_tflops"):
+            frac_measured["fp4_this_run"] = achieved / gemm["fp4_tflops"]
     roofline = {"bound": "tensor", "kernel": kern, "achieved": achieved, "peak": peaks["bf16"],
                 "unit": "TFLOP/s", "frac": achieved / peaks["bf16"], "frac_of_measured": frac_measured,
                 "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, cfg.Bc) if cfg.causal and not args.p_f32 else None),
