@@ -178,15 +178,22 @@ def measure_gemm_peaks(dev):
     return res
 
 
-def time_workload(hb, cfg, dev, steps, warmup, flush_l2, s=None, inv_s=None, qmean=False, p_f32=False, fused_q=False):
+def time_workload(hb, cfg, dev, steps, warmup, flush_l2, s=None, inv_s=None, qmean=False, p_f32=False, fused_q=False,
+                  f8qk=False):
     """Device-resident timing of one configuration: per-step time of quantize + attention (events around each
     step, L2 flushed between steps) and, from a second pass with one more event, the attention launch alone.
-    fused_q: K and V through the quantizer, Q quantized inside the attention kernel (hifa4_attention_fwd_qraw)."""
+    fused_q: K and V through the quantizer, Q quantized inside the attention kernel (hifa4_attention_fwd_qraw).
+    f8qk: the kind::f8f6f4 experiment (hifa4_attention_fwd_f8qk; its two operand-image launches count as attention)."""
     q, k, v = synth.make_qkv_device(cfg, dev)
     dt = hb._DT[q.dtype]
     qkv = hb.alloc_qkv(cfg.B, cfg.Hq, cfg.Hkv, cfg.N, cfg.d, dt, dev, qmean=qmean)
     out = torch.empty((cfg.B, cfg.Hq, cfg.N, cfg.d), dtype=torch.float32, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
+    f8_ws = None
+    if f8qk:
+        import ctypes
+        sh_ = hb._shape(cfg.B, cfg.Hq, cfg.Hkv, cfg.N, cfg.d, dt, None)
+        f8_ws = torch.empty(int(hb.lib().hifa4_f8qk_workspace_bytes(ctypes.byref(sh_))), dtype=torch.uint8, device=dev)
 
     def step(split):
         hb.quantize_qkv(None if fused_q else q, k, v, s, inv_s, out=qkv, d_status=status, qmean=qmean, Hq=cfg.Hq)
@@ -194,7 +201,9 @@ def time_workload(hb, cfg, dev, steps, warmup, flush_l2, s=None, inv_s=None, qme
         if split:
             mid = torch.cuda.Event(enable_timing=True)
             mid.record()
-        if fused_q:
+        if f8qk:
+            hb.attention_fwd_f8qk(qkv, cfg.causal, out_dtype=hb.F32, out=out, workspace=f8_ws, d_status=status)
+        elif fused_q:
             hb.attention_fwd_qraw(q, s, qkv, cfg.causal, out_dtype=hb.F32, out=out, d_status=status,
                                   p_dtype=hb.F32 if p_f32 else hb.F16)
         else:
@@ -314,6 +323,8 @@ def main():
     ap.add_argument("--p-f32", action="store_true",
                     help="variant: quantize the FP32 exponential (not the method's FP16 P; for comparison only)")
     ap.add_argument("--qmean", action="store_true", help="with the Q-Mean auxiliary (Algorithm 1 lines 2 and 6)")
+    ap.add_argument("--f8qk", action="store_true",
+                    help="experiment: Q K^T as kind::f8f6f4 with one accumulator per HIF4 group (d = 128, Bc = 64)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-context", action="store_true", help="skip the torch SDPA / N=8192 context numbers")
@@ -370,6 +381,12 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)       # > 126 MB of L2
     flush_rd = torch.zeros(64 << 20, dtype=torch.float32, device=dev)   # 256 MiB that are only read
 
+    f8_ws = None
+    if args.f8qk:
+        import ctypes
+        sh_ = hb._shape(cfg.B, cfg.Hq, cfg.Hkv, cfg.N, cfg.d, dt, None)
+        f8_ws = torch.empty(int(hb.lib().hifa4_f8qk_workspace_bytes(ctypes.byref(sh_))), dtype=torch.uint8, device=dev)
+
     def flush_l2():
         # Write a buffer larger than L2, then read another one: the write evicts every line of the
         # previous step, the read pass pushes the dirty lines of the write out to HBM, so that their
@@ -386,8 +403,11 @@ def main():
         if split:
             mid = torch.cuda.Event(enable_timing=True)
             mid.record()
-        hb.attention_fwd(qkv, cfg.causal, Bc=cfg.Bc, out_dtype=hb.F32, out=out, d_status=status,
-                         p_dtype=hb.F32 if args.p_f32 else hb.F16, qmean=args.qmean)
+        if args.f8qk:
+            hb.attention_fwd_f8qk(qkv, cfg.causal, out_dtype=hb.F32, out=out, workspace=f8_ws, d_status=status)
+        else:
+            hb.attention_fwd(qkv, cfg.causal, Bc=cfg.Bc, out_dtype=hb.F32, out=out, d_status=status,
+                             p_dtype=hb.F32 if args.p_f32 else hb.F16, qmean=args.qmean)
         return mid
 
     def barrier():
@@ -457,7 +477,7 @@ def main():
     # FP16 output (the method's final normalisation is FP16: Appendix, "FP16 operations") and FP32 output (the
     # dtype the parity tests judge); the FP16 one is the line's `e2e`.
     e2e = e2e_f32 = None
-    if not big and not args.qmean and not args.p_f32:
+    if not big and not args.qmean and not args.p_f32 and not args.f8qk:
         pq, pk, pv = qh.pin_memory(), kh.pin_memory(), vh.pin_memory()
         # One problem per batch element: hifa4_attention_fwd_raw on its Q/K/V (contiguous slices).  One stream
         # carries all host-to-device copies, one all device-to-host copies, the kernels of consecutive problems
@@ -587,7 +607,7 @@ def main():
     # device like the headline (events around each step, L2 flushed between steps), under the same clock record
     sweep, gemm, sweep_clocks = None, None, None
     headline = cfg.name == synth.CONFIGS["C2"].name and cfg.N == 4096 and cfg.causal and cfg.Bc == 64 \
-        and not args.qmean and not args.p_f32
+        and not args.qmean and not args.p_f32 and not args.f8qk
     if rank == 0 and headline and not args.no_sweep:
         gemm = measure_gemm_peaks(dev)
         del out
@@ -608,6 +628,8 @@ def main():
                    ("C2 Bc=128", synth.config("C2", Bc=128), {}),
                    ("C2 Q-Mean", synth.config("C2"), {"qmean": True}),
                    ("C2 FP32-P variant", synth.config("C2"), {"p_f32": True}),
+                   ("C2 Q K^T as kind::f8f6f4 with split accumulators (experiment; incl. 2 operand-image launches)",
+                    synth.config("C2"), {"f8qk": True}),
                    ("C2 Q quantized inside the attention kernel", synth.config("C2"), {"fused_q": True}),
                    ("C2@8192 Q quantized inside the attention kernel", synth.config("C2", N=8192), {"fused_q": True}),
                    ("C3", synth.config("C3"), {}), ("C4", synth.config("C4"), {})]
@@ -636,7 +658,9 @@ def main():
     value = whole_job_tflops(cfg, world, args.steps, total_ms)
     attn_avg_ms = sum(attn_ms) / len(attn_ms)
     achieved = fl / (attn_avg_ms * 1e-3) / 1e12
-    if cfg.Bc == 64 and cfg.d in (128, 256):
+    if args.f8qk:
+        kern = "attention_fwd_ws64_kernel<128, f8f6f4 experiment> + 2 x f8_image_kernel"
+    elif cfg.Bc == 64 and cfg.d in (128, 256):
         kern = f"attention_fwd_ws64_kernel<{cfg.d}>"
     elif cfg.Bc == 128 and cfg.d == 128:
         kern = "attention_fwd_ws_kernel<4>"

@@ -289,6 +289,23 @@ int hifa4_attention_fwd_qraw(const hifa4_shape* shape, const void* q, const floa
                              const hifa4_qkv* kv, const hifa4_attn_params* prm, void* out,
                              void* workspace, int* d_status, void* stream);
 
+/* Experiment, not a default path: hifa4_attention_fwd with S = Q-hat K-hat^T issued
+ * as tcgen05.mma kind::f8f6f4 (the 8-bit MMA kind nearest to the "HIF4 Cube" of
+ * Algorithm 1's comments).  Element x micro-exponent (an integer up to 28) is exact
+ * in E4M3; the E6M2 group scale is not, so S is accumulated separately per
+ * 64-channel group and the two partial sums are combined with the FP32 group
+ * scales by the softmax threads (exact products, one rounding).  The call first
+ * derives the E4M3 images and group scales of Q and K from qkv's packed codes and
+ * metadata into `workspace` (hifa4_f8qk_workspace_bytes(), 256-byte aligned), then
+ * runs the attention kernel; P V is unchanged (v_mma is read).  d = 128, Bc = 64,
+ * qmean = 0, normalizer = 0, p_dtype = F16; anything else returns
+ * HIFA4_ERR_UNSUPPORTED.  The result meets the same bars against the oracle as
+ * hifa4_attention_fwd (the scores are the correctly rounded exact sums). */
+size_t hifa4_f8qk_workspace_bytes(const hifa4_shape* shape);
+int hifa4_attention_fwd_f8qk(const hifa4_shape* shape, const hifa4_qkv* qkv,
+                             const hifa4_attn_params* prm, void* out, void* workspace,
+                             size_t workspace_bytes, int* d_status, void* stream);
+
 /* Workspace for hifa4_attention_fwd_raw: all hifa4_qkv buffers (each rounded up
  * to 256 bytes; the two Q-Mean vectors only when prm->qmean = 1) plus the
  * attention workspace. */

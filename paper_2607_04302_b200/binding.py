@@ -108,6 +108,11 @@ def lib():
         L.hifa4_attention_fwd_qraw.argtypes = [C.POINTER(_Shape), C.c_void_p, C.c_void_p, C.POINTER(_QKV),
                                                C.POINTER(_AttnParams), C.c_void_p, C.c_void_p, C.c_void_p,
                                                C.c_void_p]
+        L.hifa4_f8qk_workspace_bytes.restype = C.c_size_t
+        L.hifa4_f8qk_workspace_bytes.argtypes = [C.POINTER(_Shape)]
+        L.hifa4_attention_fwd_f8qk.restype = C.c_int
+        L.hifa4_attention_fwd_f8qk.argtypes = [C.POINTER(_Shape), C.POINTER(_QKV), C.POINTER(_AttnParams), C.c_void_p,
+                                               C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.hifa4_selftest_wait_timeout.restype = C.c_int
         L.hifa4_selftest_wait_timeout.argtypes = [C.POINTER(_Shape), C.POINTER(_QKV), C.POINTER(_AttnParams),
                                                   C.c_void_p, C.c_void_p, C.c_void_p]
@@ -129,7 +134,8 @@ EXPORTS = ("hifa4_status_string", "hifa4_get_counters", "hifa4_smooth_calibrate"
            "hifa4_smooth_calibrate_static", "hifa4_smooth_calibrate_auto", "hifa4_quant_bytes",
            "hifa4_quantize_qkv", "hifa4_attention_workspace_bytes", "hifa4_attention_fwd",
            "hifa4_attention_fwd_stats", "hifa4_attention_raw_workspace_bytes", "hifa4_attention_fwd_raw",
-           "hifa4_attention_fwd_qraw", "hifa4_selftest_wait_timeout")
+           "hifa4_attention_fwd_qraw", "hifa4_f8qk_workspace_bytes", "hifa4_attention_fwd_f8qk",
+           "hifa4_selftest_wait_timeout")
 
 
 def status_string(status: int) -> str:
@@ -359,6 +365,26 @@ def attention_fwd_qraw(q, s, kv: QuantizedQKV, causal: bool, out_dtype=F32, out=
     rc = lib().hifa4_attention_fwd_qraw(C.byref(sh), _ptr(q), _ptr(s), C.byref(st), C.byref(prm), _ptr(out), None,
                                         _ptr(d_status), _stream())
     _check(rc, "hifa4_attention_fwd_qraw")
+    return out
+
+
+def attention_fwd_f8qk(qkv: QuantizedQKV, causal: bool, out_dtype=F32, out=None, workspace=None, d_status=None,
+                       softmax_scale=0.0):
+    """attention_fwd with Q K^T issued as kind::f8f6f4 on E4M3 images (experiment; d = 128, Bc = 64)."""
+    dev = qkv.k_mma.device
+    sh = _shape(qkv.B, qkv.Hq, qkv.Hkv, qkv.N, qkv.d, qkv.in_dtype, qkv.q_to_kv)
+    prm = _params(causal, 64, out_dtype, softmax_scale=softmax_scale)
+    need = int(lib().hifa4_f8qk_workspace_bytes(C.byref(sh)))
+    if need == 0:
+        raise Hifa4Error(2, "hifa4_f8qk_workspace_bytes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    if out is None:
+        out = torch.empty((qkv.B, qkv.Hq, qkv.N, qkv.d), dtype=_TORCH_DT[out_dtype], device=dev)
+    st = qkv.struct()
+    rc = lib().hifa4_attention_fwd_f8qk(C.byref(sh), C.byref(st), C.byref(prm), _ptr(out), _ptr(workspace),
+                                        C.c_size_t(workspace.numel()), _ptr(d_status), _stream())
+    _check(rc, "hifa4_attention_fwd_f8qk")
     return out
 
 

@@ -208,7 +208,7 @@ size_t hifa4_attention_workspace_bytes(const hifa4_shape* shape, const hifa4_att
 static int attention_common(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
                             void* out, const hifa4_debug* dbg, const hifa4_mass_stats* stats, int* d_status,
                             void* stream, bool selftest = false, const void* q_raw = nullptr,
-                            const float* q_scale = nullptr)
+                            const float* q_scale = nullptr, const F8Operands* f8 = nullptr)
 {
     g_calls[2].fetch_add(1, std::memory_order_relaxed);
     int rc = check_attn(shape, prm);
@@ -229,7 +229,7 @@ static int attention_common(const hifa4_shape* shape, const hifa4_qkv* qkv, cons
     if ((rc = build_map(shape->Hq, shape->Hkv, shape->q_to_kv, qmap, kmap))) return rc;
     if ((rc = check_arch())) return rc;
     return launch_attention(*shape, qmap, *qkv, *prm, out, dbg, stats, d_status, (cudaStream_t)stream, selftest,
-                            q_raw, q_scale);
+                            q_raw, q_scale, f8);
 }
 
 int hifa4_attention_fwd(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,
@@ -250,6 +250,37 @@ int hifa4_attention_fwd_qraw(const hifa4_shape* shape, const void* q, const floa
     if (rc) return rc;
     if (!attention_qraw_supported(*shape, *prm)) return HIFA4_ERR_UNSUPPORTED;
     return attention_common(shape, kv, prm, out, nullptr, nullptr, d_status, stream, false, q, s);
+}
+
+size_t hifa4_f8qk_workspace_bytes(const hifa4_shape* shape)
+{
+    if (check_shape(shape) != HIFA4_OK || shape->d != 128) return 0;
+    const size_t rq = (size_t)shape->B * shape->Hq * shape->N, rk = (size_t)shape->B * shape->Hkv * shape->N;
+    return align256(rq * 128) + align256(rk * 128) + align256(rq * 2 * sizeof(float)) + align256(rk * 2 * sizeof(float));
+}
+
+int hifa4_attention_fwd_f8qk(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm, void* out,
+                             void* workspace, size_t workspace_bytes, int* d_status, void* stream)
+{
+    int rc = check_attn(shape, prm);
+    if (rc) return rc;
+    if (shape->d != 128 || prm->Bc != 64 || prm->qmean || prm->normalizer || prm->p_dtype == HIFA4_F32) return HIFA4_ERR_UNSUPPORTED;
+    if (!qkv || !out || !qkv->q_codes || !qkv->q_meta || !qkv->k_codes || !qkv->k_meta || !qkv->v_mma) return HIFA4_ERR_INVALID_ARG;
+    const size_t need = hifa4_f8qk_workspace_bytes(shape);
+    if (!workspace || workspace_bytes < need || ((uintptr_t)workspace & 255)) return HIFA4_ERR_WORKSPACE;
+    if ((rc = check_arch())) return rc;
+    const size_t rq = (size_t)shape->B * shape->Hq * shape->N, rk = (size_t)shape->B * shape->Hkv * shape->N;
+    char* base = (char*)workspace;
+    void* q_f8 = base; base += align256(rq * 128);
+    void* k_f8 = base; base += align256(rk * 128);
+    float* q_gs = (float*)base; base += align256(rq * 2 * sizeof(float));
+    float* k_gs = (float*)base;
+    if (launch_f8_images(*shape, *qkv, q_f8, q_gs, k_f8, k_gs, (cudaStream_t)stream) != cudaSuccess) return HIFA4_ERR_CUDA;
+    const F8Operands f8{q_f8, k_f8, q_gs, k_gs};
+    hifa4_qkv tmp = *qkv;
+    if (!tmp.q_mma) tmp.q_mma = q_f8;                       // not read by this launch; the common check wants non-null
+    if (!tmp.k_mma) tmp.k_mma = k_f8;
+    return attention_common(shape, &tmp, prm, out, nullptr, nullptr, d_status, stream, false, nullptr, nullptr, &f8);
 }
 
 int hifa4_selftest_wait_timeout(const hifa4_shape* shape, const hifa4_qkv* qkv, const hifa4_attn_params* prm,

@@ -325,6 +325,19 @@ bool make_bf16_map(CUtensorMap* m, void* base, uint64_t heads, uint64_t rows, ui
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_u8_map(CUtensorMap* m, void* base, uint64_t heads, uint64_t rows, uint64_t cols, uint32_t box_rows)
+{
+    EncodeTiledFn enc = get_encode();
+    if (!enc || cols != 128) return false;                 // one 128-byte swizzle span per row
+    cuuint64_t dims[3] = {cols, rows, heads};
+    cuuint64_t strides[2] = {cols, rows * cols};
+    cuuint32_t box[3] = {128, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int D, int BC, bool AUX>
 static int launch_cfg(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
@@ -350,10 +363,16 @@ bool attention_qraw_supported(const hifa4_shape& sh, const hifa4_attn_params& pr
 int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv& qkv,
                      const hifa4_attn_params& prm, void* out, const hifa4_debug* dbg,
                      const hifa4_mass_stats* stats, int* d_status, cudaStream_t st, bool selftest,
-                     const void* q_raw, const float* q_scale)
+                     const void* q_raw, const float* q_scale, const F8Operands* f8)
 {
     AttnArgs a;
     memset(&a, 0, sizeof(a));
+    if (f8) {
+        if (prm.Bc != 64 || sh.d != 128 || prm.qmean || prm.normalizer || prm.p_dtype == HIFA4_F32 || stats || selftest ||
+            q_raw || (dbg && dbg->n_blocks > 0))
+            return HIFA4_ERR_UNSUPPORTED;
+        a.q_f8 = f8->q_f8; a.k_f8 = f8->k_f8; a.q_gs = f8->q_gs; a.k_gs = f8->k_gs;
+    }
     if (q_raw) {
         if (!attention_qraw_supported(sh, prm) || stats || selftest || (dbg && dbg->n_blocks > 0)) return HIFA4_ERR_UNSUPPORTED;
         a.q_raw = q_raw;

@@ -33,6 +33,9 @@ struct AttnArgs {
     int qmean;                    // add mu_i * k_sum_j to the raw scores (Algorithm 1 line 6)
     const float* q_mu;            // [B,Hq,N]
     const float* k_sum;           // [B,Hkv,N]
+    // kind::f8f6f4 experiment (Q K^T on E4M3 images of element x micro-exponent, one accumulator per 64-channel group)
+    const void *q_f8, *k_f8;      // [B,H,N,d] bytes, else null
+    const float *q_gs, *k_gs;     // [B,H,N,d/64] group scales S/4
     const void* q_raw;            // raw-Q launch (Q is quantized inside the kernel): the 16-bit Q [B,Hq,N,d], else null
     const float* q_scale;         // raw-Q launch: Smooth-QK factors of Q [Hkv,d] or null
     int in_dtype;                 // raw-Q launch: HIFA4_F16 or HIFA4_BF16

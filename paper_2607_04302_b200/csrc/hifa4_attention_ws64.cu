@@ -42,31 +42,37 @@
 
 namespace hifa4 {
 
-template <int D_>
+// F8: the kind::f8f6f4 experiment (d = 128): Q and K tiles are one byte per element, S has one accumulator per
+// 64-channel group, 304 tensor-memory columns, hence one CTA per SM.
+template <int D_, bool F8 = false>
 struct WS64 {
     static constexpr int D = D_, BC = 64, STAGES = 2;
     static constexpr int NSW = 8, THREADS = (NSW + 2) * 32, W_QK = NSW, W_PV = NSW + 1;   // two groups of 4 softmax warps
     static constexpr int NU = BC / 8;                       // 8 level-2 units (64 keys) per thread and tile
     static constexpr int QSUB = D / 64;                     // 64-channel sub-tiles of Q and K
-    static constexpr int Q_BYTES = QSUB * 16384;
+    static constexpr int Q_BYTES = F8 ? 128 * D : QSUB * 16384;
     static constexpr int K_SUB = BC * 128;                  // 64 keys x 64 channels
-    static constexpr int K_STAGE = QSUB * K_SUB;
+    static constexpr int K_STAGE = F8 ? BC * D : QSUB * K_SUB;
     static constexpr int V_STAGE = (D + 16) * 128;          // D rows of V^T + 16 rows of ones, 64 keys wide
     static constexpr int Q_OFF = 0;
     static constexpr int K_OFF = Q_OFF + Q_BYTES;
     static constexpr int V_OFF = K_OFF + STAGES * K_STAGE;
     static constexpr int MISC_OFF = V_OFF + STAGES * V_STAGE;
     static constexpr int KSUM_SLOTS = 4;                    // Q-Mean: channel sums of a tile's 64 keys; slot = tile % 4
+    static constexpr int KSUM_BYTES = F8 ? 512 : 256;       // (F8: the two group scales of each of the tile's keys instead)
     static constexpr int KSUM_OFF = MISC_OFF + 256;
-    static constexpr int MX_OFF = KSUM_OFF + KSUM_SLOTS * 256;  // running maxima handed from tile j to tile j+1: [2][128] floats
-    static constexpr int SMEM_BYTES = MX_OFF + 2 * 512 + 1024;
+    static constexpr int MX_OFF = KSUM_OFF + KSUM_SLOTS * KSUM_BYTES;  // running maxima handed from tile j to tile j+1: [2][128] floats
+    static constexpr int SMEM_USED = MX_OFF + 2 * 512 + 1024;
+    // F8 allocates all 512 tensor-memory columns: it asks for more than half of the SM's shared memory as well, so
+    // that a second CTA never becomes resident only to block in the tensor-memory allocator
+    static constexpr int SMEM_BYTES = (F8 && SMEM_USED < 120 * 1024) ? 120 * 1024 : SMEM_USED;
     static constexpr int O_COLS = D + 16;
     static constexpr bool Q_IN_TMEM = (D == 256);
     static constexpr int QT_COL = 272;                      // d = 256 only
     static constexpr int S_COL = (D == 256) ? 400 : 144;
-    static constexpr int P_COL = S_COL + 64;
-    static constexpr int TMEM_COLS = (D == 256) ? 512 : 256;
-    static constexpr int CTAS_PER_SM = (D == 256) ? 1 : 2;
+    static constexpr int P_COL = S_COL + (F8 ? 128 : 64);
+    static constexpr int TMEM_COLS = (D == 256 || F8) ? 512 : 256;
+    static constexpr int CTAS_PER_SM = (D == 256 || F8) ? 1 : 2;
 };
 namespace ws64 {
 // Index s = tile % 2 everywhere.  QKGO[s]: K stage s has landed and S is free (4 arrivals + 1 + bytes); PVGO[s]:
@@ -106,14 +112,19 @@ static __device__ __forceinline__ void arrive_lane0(uint32_t bar, int lane)
 // has landed and no MMA is in flight, so the CTA leaves through the ordinary failure exit.
 // QRAW: the Q tensor map is over the raw 16-bit Q; the softmax threads smooth and HIF4-quantize their CTA's 128 rows
 // in shared memory (Algorithm 1 line 1) before the first S = Q K^T, so Q-hat never travels through HBM.
-template <int DH, bool DBG, bool PF32, bool QM, bool SELFTEST = false, bool QRAW = false>
-__global__ void __launch_bounds__(WS64<DH>::THREADS, WS64<DH>::CTAS_PER_SM)
+// F8QK: the kind::f8f6f4 experiment.  Q-hat and K-hat arrive as E4M3 images of element x micro-exponent (integers up
+// to 28, exact) with one FP32 scale S/4 per (row, 64-channel group); S = Q K^T runs as two accumulators, one per
+// channel group, and the softmax threads bind them: acc = (qs0 ks0_j) S0 + (qs1 ks1_j) S1, every product exact and
+// the sum rounded once.  Measured against the BF16-image form, not a default path.
+template <int DH, bool DBG, bool PF32, bool QM, bool SELFTEST = false, bool QRAW = false, bool F8QK = false>
+__global__ void __launch_bounds__(WS64<DH, F8QK>::THREADS, WS64<DH, F8QK>::CTAS_PER_SM)
 attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                            const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ AttnArgs args)
 {
     using namespace ws64;
-    using C = WS64<DH>;
+    using C = WS64<DH, F8QK>;
     static_assert(!QRAW || (DH == 128 && !QM && !DBG), "raw-Q launch: d = 128, no Q-Mean, no dump");
+    static_assert(!F8QK || (DH == 128 && !QM && !DBG && !QRAW && !SELFTEST), "f8f6f4 experiment: d = 128, plain path");
     constexpr int D = C::D, BC = C::BC, STAGES = C::STAGES, NSW = C::NSW, THREADS = C::THREADS;
     constexpr int W_QK = C::W_QK, W_PV = C::W_PV, NU = C::NU, QSUB = C::QSUB;
     constexpr int Q_BYTES = C::Q_BYTES, K_SUB = C::K_SUB, K_STAGE = C::K_STAGE, V_STAGE = C::V_STAGE;
@@ -149,9 +160,16 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     auto load_k = [&](int jt) {                               // K tile jt into stage jt % 2
         const int st = jt & 1;
         mbar_expect_tx(bar(BAR_QKGO + st), K_STAGE);
+        if constexpr (F8QK) {
+            tma_load_3d(k_s + st * K_STAGE, &tmap_k, bar(BAR_QKGO + st), 0, jt * BC, bh_kv);
+            // the tile's 64 x 2 key group scales: four slots with a barrier each, as the Q-Mean key sums below
+            mbar_expect_tx(bar(BAR_KSF + (jt & 3)), 512);
+            bulk_load(smem_base + C::KSUM_OFF + (jt & 3) * 512, args.k_gs + ((size_t)bh_kv * N + jt * BC) * 2, 512, bar(BAR_KSF + (jt & 3)));
+        } else {
 #pragma unroll
-        for (int s = 0; s < QSUB; ++s)
-            tma_load_3d(k_s + st * K_STAGE + s * K_SUB, &tmap_k, bar(BAR_QKGO + st), 64 * s, jt * BC, bh_kv);
+            for (int s = 0; s < QSUB; ++s)
+                tma_load_3d(k_s + st * K_STAGE + s * K_SUB, &tmap_k, bar(BAR_QKGO + st), 64 * s, jt * BC, bh_kv);
+        }
         if (QM) {
             // Q-Mean: the 64 channel sums of this tile's keys travel with the K tile, two tiles ahead of their use
             // right after S is pulled (with the V^T tile they arrived ~2000 clk after the softmax warps wanted
@@ -193,8 +211,12 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         *abort_flag = status_now != 0 ? 2 : 0;
         if (status_now == 0) {
             mbar_expect_tx(bar(BAR_Q), Q_BYTES);
+            if constexpr (F8QK) {
+                tma_load_3d(q_s, &tmap_q, bar(BAR_Q), 0, q0, bh_q);
+            } else {
 #pragma unroll
-            for (int s = 0; s < QSUB; ++s) tma_load_3d(q_s + s * 16384, &tmap_q, bar(BAR_Q), 64 * s, q0, bh_q);
+                for (int s = 0; s < QSUB; ++s) tma_load_3d(q_s + s * 16384, &tmap_q, bar(BAR_Q), 64 * s, q0, bh_q);
+            }
             load_k(0);
             if (n_tiles > 1) load_k(1);
         }
@@ -233,11 +255,18 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 if (!wait64(bar(BAR_QKGO + st), ph, abort_flag)) { fail(4); break; }
                 tc_fence_after();
                 const uint32_t b0 = k_lo + st * (K_STAGE >> 4);
+                if constexpr (F8QK) {
+                    constexpr uint32_t idesc_f8 = umma_idesc_e4m3(128, BC);
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {          // D / 16 steps of 16 channels
-                    const uint32_t kb = b0 + (kk >> 2) * (K_SUB >> 4) + (kk & 3) * 2;
-                    if constexpr (C::Q_IN_TMEM) umma_bf16_ts_lo(tmem + S_COL, tmem + QT_COL + kk * 8, kb, idesc_s, kk ? 1u : 0u);
-                    else umma_bf16_ss_lo(tmem + S_COL, q_lo + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2, kb, idesc_s, kk ? 1u : 0u);
+                    for (int kk = 0; kk < 4; ++kk)             // 32 channels per step; steps 0, 1 -> S0, steps 2, 3 -> S1
+                        umma_f8_ss_lo(tmem + S_COL + (kk >> 1) * 64, q_lo + kk * 2, b0 + kk * 2, idesc_f8, kk & 1);
+                } else {
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {      // D / 16 steps of 16 channels
+                        const uint32_t kb = b0 + (kk >> 2) * (K_SUB >> 4) + (kk & 3) * 2;
+                        if constexpr (C::Q_IN_TMEM) umma_bf16_ts_lo(tmem + S_COL, tmem + QT_COL + kk * 8, kb, idesc_s, kk ? 1u : 0u);
+                        else umma_bf16_ss_lo(tmem + S_COL, q_lo + (kk >> 2) * (16384 >> 4) + (kk & 3) * 2, kb, idesc_s, kk ? 1u : 0u);
+                    }
                 }
                 umma_commit(bar(BAR_SF + st));
                 umma_commit(bar(BAR_KE + st));
@@ -291,6 +320,11 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                 if (args.dbg.blocks[3 * i] == b && args.dbg.blocks[3 * i + 1] == h && args.dbg.blocks[3 * i + 2] == qt)
                     dbg_slot = i;
         const float mu_row = (QM && row < N) ? args.q_mu[(size_t)bh_q * N + row] : 0.f;
+        float qs0 = 0.f, qs1 = 0.f;                                 // f8f6f4 experiment: the row's two group scales
+        if (F8QK && row < N) {
+            qs0 = args.q_gs[((size_t)bh_q * N + row) * 2];
+            qs1 = args.q_gs[((size_t)bh_q * N + row) * 2 + 1];
+        }
         float* mx_s = reinterpret_cast<float*>(smem_gen + C::MX_OFF);   // [2][128]
         float m_run = -INFINITY;
         bool ok = true;
@@ -340,7 +374,27 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             if (!wait64(bar(BAR_SF + st), ph, abort_flag)) { fail(8); ok = false; break; }
             tc_fence_after();
             float p[BC];
-            {
+            if constexpr (F8QK) {
+                // bind the two per-group integer sums: acc = (qs0 ks0_j) S0 + (qs1 ks1_j) S1.  The scales have 3
+                // significant bits, the sums at most 16: both products are exact, the sum is rounded once.
+                if (!wait64(bar(BAR_KSF + (jt & 3)), (uint32_t)(jt >> 2) & 1u, abort_flag)) { fail(15); ok = false; break; }
+                const uint32_t ks_s = smem_base + C::KSUM_OFF + (jt & 3) * 512;
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {               // 32 keys at a time
+                    uint32_t r0[32], r1[32];
+                    tmem_ld32(t_lane + S_COL + 32 * hh, r0);
+                    tmem_ld32(t_lane + S_COL + 64 + 32 * hh, r1);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        float4 ks;                             // ks0_j, ks1_j, ks0_{j+1}, ks1_{j+1}
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                     : "=f"(ks.x), "=f"(ks.y), "=f"(ks.z), "=f"(ks.w) : "r"(ks_s + 8 * (32 * hh + i)));
+                        p[32 * hh + i] = fmaf(qs1 * ks.y, __uint_as_float(r1[i]), (qs0 * ks.x) * __uint_as_float(r0[i]));
+                        p[32 * hh + i + 1] = fmaf(qs1 * ks.w, __uint_as_float(r1[i + 1]), (qs0 * ks.z) * __uint_as_float(r0[i + 1]));
+                    }
+                }
+            } else {
                 uint32_t r[BC];
                 tmem_ld32(t_lane + S_COL, reinterpret_cast<uint32_t(&)[32]>(r[0]));
                 tmem_ld32(t_lane + S_COL + 32, reinterpret_cast<uint32_t(&)[32]>(r[32]));
@@ -540,15 +594,22 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     if (warp == W_QK) { __syncwarp(); tmem_dealloc(tmem, TMEM_COLS); }
 }
 
-template <int DH, bool DBG, bool PF32, bool QM, bool SELFTEST = false, bool QRAW = false>
+bool make_u8_map(CUtensorMap* m, void* base, uint64_t heads, uint64_t rows, uint64_t cols, uint32_t box_rows);
+
+template <int DH, bool DBG, bool PF32, bool QM, bool SELFTEST = false, bool QRAW = false, bool F8QK = false>
 static int launch_ws64(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
-    using C = WS64<DH>;
+    using C = WS64<DH, F8QK>;
     CUtensorMap mq, mk, mv;
-    if (!make_bf16_map(&mq, QRAW ? const_cast<void*>(args.q_raw) : qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, DH, 128)) return HIFA4_ERR_CUDA;
-    if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, DH, C::BC)) return HIFA4_ERR_CUDA;
+    if constexpr (F8QK) {
+        if (!make_u8_map(&mq, const_cast<void*>(args.q_f8), (uint64_t)sh.B * sh.Hq, sh.N, DH, 128)) return HIFA4_ERR_CUDA;
+        if (!make_u8_map(&mk, const_cast<void*>(args.k_f8), (uint64_t)sh.B * sh.Hkv, sh.N, DH, C::BC)) return HIFA4_ERR_CUDA;
+    } else {
+        if (!make_bf16_map(&mq, QRAW ? const_cast<void*>(args.q_raw) : qkv.q_mma, (uint64_t)sh.B * sh.Hq, sh.N, DH, 128)) return HIFA4_ERR_CUDA;
+        if (!make_bf16_map(&mk, qkv.k_mma, (uint64_t)sh.B * sh.Hkv, sh.N, DH, C::BC)) return HIFA4_ERR_CUDA;
+    }
     if (!make_bf16_map(&mv, qkv.v_mma, (uint64_t)sh.B * sh.Hkv, DH, sh.N, DH)) return HIFA4_ERR_CUDA;
-    auto kern = attention_fwd_ws64_kernel<DH, DBG, PF32, QM, SELFTEST, QRAW>;
+    auto kern = attention_fwd_ws64_kernel<DH, DBG, PF32, QM, SELFTEST, QRAW, F8QK>;
     static SmemOptIn opt_in;
     if (!opt_in.ensure(kern, C::SMEM_BYTES)) return HIFA4_ERR_CUDA;
     dim3 grid((unsigned)(((sh.N + 127) / 128) * sh.Hq * sh.B));
@@ -571,6 +632,13 @@ template <int DH>
 static int launch_ws64_d(const hifa4_shape& sh, const hifa4_qkv& qkv, const AttnArgs& args, cudaStream_t st)
 {
     const bool dbg = args.dbg.n_blocks > 0;
+    if (args.q_f8) {                                       // the kind::f8f6f4 experiment: d = 128, plain path only
+        if constexpr (DH != 128) return HIFA4_ERR_UNSUPPORTED;
+        else {
+            if (dbg || args.qmean || args.p_f32 || args.q_raw) return HIFA4_ERR_UNSUPPORTED;
+            return launch_ws64<DH, false, false, false, false, false, true>(sh, qkv, args, st);
+        }
+    }
     if (args.q_raw) {                                      // Q quantized in the kernel: d = 128, no Q-Mean, no dump
         if constexpr (DH != 128) return HIFA4_ERR_UNSUPPORTED;
         else {

@@ -51,10 +51,18 @@ const double* gate_result(void* gate_ws);
 // Attention forward on the BF16 operand images; returns a hifa4_status.
 // q_raw non-null: Q is the raw 16-bit tensor (qkv.q_mma is not read) and is smoothed with q_scale (or not, if null)
 // and quantized inside the kernel; see attention_qraw_supported.
+// Operands of the kind::f8f6f4 experiment: E4M3 images of element x micro-exponent and the per-group scales S/4.
+struct F8Operands {
+    const void *q_f8, *k_f8;      // [B,H,N,d] bytes
+    const float *q_gs, *k_gs;     // [B,H,N,d/64]
+};
+// From the packed codes and metadata of Q and K (either may be null).
+cudaError_t launch_f8_images(const hifa4_shape& sh, const hifa4_qkv& qkv, void* q_f8, float* q_gs, void* k_f8, float* k_gs,
+                             cudaStream_t st);
 int launch_attention(const hifa4_shape& shape, const HeadMap& map, const hifa4_qkv& qkv,
                      const hifa4_attn_params& prm, void* out, const hifa4_debug* dbg,
                      const hifa4_mass_stats* stats, int* d_status, cudaStream_t st, bool selftest = false,
-                     const void* q_raw = nullptr, const float* q_scale = nullptr);
+                     const void* q_raw = nullptr, const float* q_scale = nullptr, const F8Operands* f8 = nullptr);
 // Configurations whose attention kernel can quantize Q itself: the 64-key kernel for d = 128 (256 softmax threads =
 // 128 rows x two 64-channel groups) in its default arithmetic or the FP32-P variant, without Q-Mean (the row mean
 // needs the whole row before any group is quantized).

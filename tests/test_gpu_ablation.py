@@ -177,3 +177,36 @@ def test_method_components_against_fp32_attention(hb, par, N):
     # radial contraction of the mismatched output: its projection on the consistent one is below 1
     shrink = float((o_smooth_mis * o_hifa4).sum() / (o_hifa4 * o_hifa4).sum())
     assert 0.85 < shrink < 0.99, shrink
+
+
+@pytest.mark.parametrize("shape", [dict(B=1, Hq=2, Hkv=1, N=256), dict(B=2, Hq=4, Hkv=2, N=1024, causal=False),
+                                   dict(B=1, Hq=4, Hkv=1, N=576, dtype="fp16"), dict()])
+def test_f8f6f4_score_product_is_bit_identical(hb, par, shape):
+    """The kind::f8f6f4 experiment: S = Q-hat K-hat^T on E4M3 images of element x micro-exponent, one accumulator per
+    64-channel group, the E6M2 group scales applied by the softmax threads.  Every product and both partial sums are
+    exact and the final sum is rounded once, which is also what the BF16-image MMA delivers (its products are exact
+    and its FP32 accumulation of at most 128 of them loses nothing here), so the output must equal that of
+    hifa4_attention_fwd bit for bit - and that one stands under the oracle comparison.  Last case: the headline shape."""
+    cfg = synth.config("C2", **shape)
+    q, k, v = synth.make_qkv_device(cfg, DEV)
+    s, inv_s = par.calibrate(cfg, DEV)
+    qkv = hb.quantize_qkv(q, k, v, s, inv_s)
+    want = hb.attention_fwd(qkv, cfg.causal)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    got = hb.attention_fwd_f8qk(qkv, cfg.causal, d_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(got, want)
+    got16 = hb.attention_fwd_f8qk(qkv, cfg.causal, out_dtype=hb.F16)
+    assert torch.equal(got16, hb.attention_fwd(qkv, cfg.causal, out_dtype=hb.F16))
+
+
+def test_f8f6f4_experiment_refuses_other_shapes(hb, par):
+    cfg = synth.config("C3", N=128, Hq=1, Hkv=1, d=64)
+    qkv = hb.quantize_qkv(*(t.to(DEV) for t in synth.make_qkv(cfg)))
+    with pytest.raises(hb.Hifa4Error):
+        hb.attention_fwd_f8qk(qkv, True)
+    cfg = synth.config("C2", B=1, Hq=2, Hkv=1, N=256)
+    qkv = hb.quantize_qkv(*(t.to(DEV) for t in synth.make_qkv(cfg)))
+    with pytest.raises(hb.Hifa4Error):                                   # undersized workspace
+        hb.attention_fwd_f8qk(qkv, True, workspace=torch.empty(4096, dtype=torch.uint8, device=DEV))
