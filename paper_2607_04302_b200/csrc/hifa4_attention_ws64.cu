@@ -58,7 +58,7 @@ struct WS64 {
     static constexpr int K_OFF = Q_OFF + Q_BYTES;
     static constexpr int V_OFF = K_OFF + STAGES * K_STAGE;
     static constexpr int MISC_OFF = V_OFF + STAGES * V_STAGE;
-    static constexpr int KSUM_SLOTS = 4;                    // Q-Mean: channel sums of a tile's 64 keys; slot = tile % 4
+    static constexpr int KSUM_SLOTS = 8;                    // Q-Mean: channel sums of a tile's 64 keys; slot = tile % 8
     static constexpr int KSUM_BYTES = F8 ? 512 : 256;       // (F8: the two group scales of each of the tile's keys instead)
     static constexpr int KSUM_OFF = MISC_OFF + 256;
     static constexpr int MX_OFF = KSUM_OFF + KSUM_SLOTS * KSUM_BYTES;  // running maxima handed from tile j to tile j+1: [2][128] floats
@@ -78,11 +78,11 @@ namespace ws64 {
 // Index s = tile % 2 everywhere.  QKGO[s]: K stage s has landed and S is free (4 arrivals + 1 + bytes); PVGO[s]:
 // V^T stage s has landed, the image of P-hat is stored and [O | l] rescaled (4 arrivals + 1 + bytes); KE / VE:
 // stage free (MMA commit); SF[s]: S complete; PV[s]: P V complete; MR[s]: running maxima after the tile
-// published (4 arrivals); KSF[tile % 4]: Q-Mean key sums landed (a barrier per slot); QT: Q-hat image copied to tensor memory.
+// published (4 arrivals); KSF[tile % 8]: Q-Mean key sums landed (a barrier per slot); QT: Q-hat image copied to tensor memory.
 // Two barriers per kind because each group of softmax warps sees every second tile only: a parity wait
 // must observe every phase of its barrier.
 enum { BAR_Q = 0, BAR_QKGO = 1, BAR_KE = 3, BAR_PVGO = 5, BAR_VE = 7, BAR_SF = 9, BAR_PV = 11, BAR_KSF = 13,
-       BAR_MR = 17, BAR_QT = 19, N_BARS = 20 };
+       BAR_MR = 21, BAR_QT = 23, N_BARS = 24 };
 constexpr uint32_t WAIT_POLLS = 1u << 20;
 }  // namespace ws64
 
@@ -162,9 +162,9 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         mbar_expect_tx(bar(BAR_QKGO + st), K_STAGE);
         if constexpr (F8QK) {
             tma_load_3d(k_s + st * K_STAGE, &tmap_k, bar(BAR_QKGO + st), 0, jt * BC, bh_kv);
-            // the tile's 64 x 2 key group scales: four slots with a barrier each, as the Q-Mean key sums below
-            mbar_expect_tx(bar(BAR_KSF + (jt & 3)), 512);
-            bulk_load(smem_base + C::KSUM_OFF + (jt & 3) * 512, args.k_gs + ((size_t)bh_kv * N + jt * BC) * 2, 512, bar(BAR_KSF + (jt & 3)));
+            // the tile's 64 x 2 key group scales: eight slots with a barrier each, as the Q-Mean key sums below
+            mbar_expect_tx(bar(BAR_KSF + (jt & 7)), 512);
+            bulk_load(smem_base + C::KSUM_OFF + (jt & 7) * 512, args.k_gs + ((size_t)bh_kv * N + jt * BC) * 2, 512, bar(BAR_KSF + (jt & 7)));
         } else {
 #pragma unroll
             for (int s = 0; s < QSUB; ++s)
@@ -173,12 +173,13 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
         if (QM) {
             // Q-Mean: the 64 channel sums of this tile's keys travel with the K tile, two tiles ahead of their use
             // right after S is pulled (with the V^T tile they arrived ~2000 clk after the softmax warps wanted
-            // them).  Four slots with a barrier each: slot jt % 4 held the sums of tile jt-4, whose readers arrived
-            // on the barrier that released S(jt-3) only after reading them, and this load follows S(jt-2).  (Two
-            // barriers would not do: the sums of tile jt+2 can land before a late reader has looked for those of
-            // tile jt, and a parity wait that is two phases behind never returns.)
-            mbar_expect_tx(bar(BAR_KSF + (jt & 3)), 256);
-            bulk_load(smem_base + C::KSUM_OFF + (jt & 3) * 256, args.k_sum + (size_t)bh_kv * N + jt * BC, 256, bar(BAR_KSF + (jt & 3)));
+            // them).  Eight slots with a barrier each: slot jt % 8 held the sums of tile jt-8, and this load follows
+            // S(jt-2), which was released by the group that owns tile jt-3 after it had pulled S(jt-3), which was
+            // released by the owners of tile jt-4 - the group that read the slot during tile jt-8 and has finished
+            // three tiles since.  (Two barriers by tile parity would not do: the sums of tile jt+2 can land before a
+            // late reader has looked for those of tile jt, and a parity wait that is two phases behind never returns.)
+            mbar_expect_tx(bar(BAR_KSF + (jt & 7)), 256);
+            bulk_load(smem_base + C::KSUM_OFF + (jt & 7) * 256, args.k_sum + (size_t)bh_kv * N + jt * BC, 256, bar(BAR_KSF + (jt & 7)));
         }
     };
     auto load_v = [&](int jt) {                               // V^T tile jt into stage jt % 2
@@ -199,7 +200,8 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             mbar_init(bar(BAR_QKGO + s), 5); mbar_init(bar(BAR_KE + s), 1);
             mbar_init(bar(BAR_PVGO + s), 5); mbar_init(bar(BAR_VE + s), 1);
             mbar_init(bar(BAR_SF + s), 1); mbar_init(bar(BAR_PV + s), 1);
-            mbar_init(bar(BAR_KSF + s), 1); mbar_init(bar(BAR_KSF + 2 + s), 1); mbar_init(bar(BAR_MR + s), 4);
+            for (int t = 0; t < 4; ++t) mbar_init(bar(BAR_KSF + 2 * t + s), 1);
+            mbar_init(bar(BAR_MR + s), 4);
         }
         mbar_init(bar(BAR_QT), NSW);
         fence_barrier_init();
@@ -377,8 +379,8 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             if constexpr (F8QK) {
                 // bind the two per-group integer sums: acc = (qs0 ks0_j) S0 + (qs1 ks1_j) S1.  The scales have 3
                 // significant bits, the sums at most 16: both products are exact, the sum is rounded once.
-                if (!wait64(bar(BAR_KSF + (jt & 3)), (uint32_t)(jt >> 2) & 1u, abort_flag)) { fail(15); ok = false; break; }
-                const uint32_t ks_s = smem_base + C::KSUM_OFF + (jt & 3) * 512;
+                if (!wait64(bar(BAR_KSF + (jt & 7)), (uint32_t)(jt >> 3) & 1u, abort_flag)) { fail(15); ok = false; break; }
+                const uint32_t ks_s = smem_base + C::KSUM_OFF + (jt & 7) * 512;
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {               // 32 keys at a time
                     uint32_t r0[32], r1[32];
@@ -404,11 +406,11 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
             }
             tc_fence_before();                                 // S(jt) is in registers: S(jt+1) may overwrite it
             __syncwarp();
-            if (!QM && jt + 1 < n_tiles) arrive_lane0(bar(BAR_QKGO + (st ^ 1)), lane);
+            if (jt + 1 < n_tiles) arrive_lane0(bar(BAR_QKGO + (st ^ 1)), lane);
 
             if (QM) {                                          // Q-Mean correction (line 6): + mu_i * sum_c k~_jc
-                if (!wait64(bar(BAR_KSF + (jt & 3)), (uint32_t)(jt >> 2) & 1u, abort_flag)) { fail(15); ok = false; break; }
-                const uint32_t ks_s = smem_base + C::KSUM_OFF + (jt & 3) * 256;
+                if (!wait64(bar(BAR_KSF + (jt & 7)), (uint32_t)(jt >> 3) & 1u, abort_flag)) { fail(15); ok = false; break; }
+                const uint32_t ks_s = smem_base + C::KSUM_OFF + (jt & 7) * 256;
                 const uint64_t mu2 = pack2(mu_row, mu_row);
 #pragma unroll
                 for (int i = 0; i < BC / 4; ++i) {
@@ -418,8 +420,6 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
                     unpack2(fma2(mu2, pack2(ks.x, ks.y), pack2(p[4 * i], p[4 * i + 1])), p[4 * i], p[4 * i + 1]);
                     unpack2(fma2(mu2, pack2(ks.z, ks.w), pack2(p[4 * i + 2], p[4 * i + 3])), p[4 * i + 2], p[4 * i + 3]);
                 }
-                __syncwarp();                                  // the slot has been read: only now may S(jt+1) go
-                if (jt + 1 < n_tiles) arrive_lane0(bar(BAR_QKGO + (st ^ 1)), lane);
             }
             if ((args.causal && (j0 + BC - 1 > q0)) || (j0 + BC > N)) {   // masked scores become -inf: exp gives exact zeros
 #pragma unroll
