@@ -397,9 +397,16 @@ int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv&
         a.dbg.p_codes = dbg->p_codes; a.dbg.p_step = dbg->p_step;
         a.dbg.l_out = dbg->l_out; a.dbg.m_out = dbg->m_out;
     }
-    // Head-major order pays once the K-hat and V-hat^T images of all KV heads exceed L2 (126 MB) well:
-    // measured on B = 4, Hkv = 8, d = 128: slower at N = 8192 (134 MB), +4 % at 16384, +7 % at 32768.
-    a.head_major = (double)sh.B * sh.Hkv * sh.N * sh.d * 4.0 > 200e6 ? 1 : 0;
+    // Head-major order (all query blocks of a head together, so that the CTAs in flight share the K-hat / V-hat^T
+    // images of one or two heads) pays once those images of all KV heads no longer sit in L2 (126 MB) together.
+    // Non-causal items are all equal, so the order costs no balance and wins from 67 MB up (measured on B = 4,
+    // Hkv = 8, d = 128: +4 % at N = 4096, +13 % at N = 8192 (134 MB); no difference at 33 MB and below).  Causal
+    // grids lose their global heaviest-first order with it: -10 % at 33 and 67 MB, +2 % at 134 MB, +4 % at 268 MB,
+    // +7 % at 537 MB.
+    {
+        const double kv_bytes = (double)sh.B * sh.Hkv * sh.N * sh.d * 4.0;
+        a.head_major = kv_bytes > (prm.causal ? 120e6 : 50e6) ? 1 : 0;
+    }
     a.normalizer = prm.normalizer ? 1 : 0;
     a.p_f32 = prm.p_dtype == HIFA4_F32 ? 1 : 0;
     if (selftest) {                               // the instantiation whose wait for P V runs out
