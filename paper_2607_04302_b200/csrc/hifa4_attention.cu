@@ -397,15 +397,29 @@ int launch_attention(const hifa4_shape& sh, const HeadMap& map, const hifa4_qkv&
         a.dbg.p_codes = dbg->p_codes; a.dbg.p_step = dbg->p_step;
         a.dbg.l_out = dbg->l_out; a.dbg.m_out = dbg->m_out;
     }
-    // Head-major order (all query blocks of a head together, so that the CTAs in flight share the K-hat / V-hat^T
-    // images of one or two heads) pays once those images of all KV heads no longer sit in L2 (126 MB) together.
-    // Non-causal items are all equal, so the order costs no balance and wins from 67 MB up (measured on B = 4,
-    // Hkv = 8, d = 128: +4 % at N = 4096, +13 % at N = 8192 (134 MB); no difference at 33 MB and below).  Causal
-    // grids lose their global heaviest-first order with it: -10 % at 33 and 67 MB, +2 % at 134 MB, +4 % at 268 MB,
-    // +7 % at 537 MB.
+    // CTA order of the 64-key kernel: groups of KV heads whose K-hat / V-hat^T images fit in L2 (126 MB) together with
+    // room to spare, one group after the other, so that the CTAs in flight share them; inside a group the grid keeps
+    // its heaviest-first order.  Causal: the largest divisor of B * Hkv whose images stay within 48 MB (measured on
+    // B = 4, Hq = 32, Hkv = 8, d = 128 against one group: +6 % at N = 8192, +5 % at 16384, +1 % at 32768, where
+    // single heads, which lose the heaviest-first order across heads, were the earlier choice; no change where
+    // everything fits).  Non-causal items are all equal, so nothing is lost by the smallest group: one KV head at a
+    // time once the images exceed 50 MB (+4 % at 67 MB, +15 % at 134 MB; no difference below).
     {
-        const double kv_bytes = (double)sh.B * sh.Hkv * sh.N * sh.d * 4.0;
-        a.head_major = kv_bytes > (prm.causal ? 120e6 : 50e6) ? 1 : 0;
+        const double per_kv_head = (double)sh.N * sh.d * 4.0;
+        const int n_kv = sh.B * sh.Hkv;
+        int want = prm.causal ? (int)(48e6 / per_kv_head) : (per_kv_head * n_kv > 50e6 ? 1 : n_kv);
+        if (want < 1) want = 1;
+        if (sh.q_to_kv || sh.Hq % sh.Hkv) {              // custom head map: whole batch elements only
+            int g_b = 1;
+            for (int c = 1; c <= sh.B && c * sh.Hkv <= want; ++c)
+                if (sh.B % c == 0) g_b = c;
+            a.group_heads = g_b * sh.Hq;
+        } else {
+            int g_kv = 1;
+            for (int c = 1; c <= n_kv && c <= want; ++c)
+                if (n_kv % c == 0) g_kv = c;
+            a.group_heads = g_kv * (sh.Hq / sh.Hkv);
+        }
     }
     a.normalizer = prm.normalizer ? 1 : 0;
     a.p_f32 = prm.p_dtype == HIFA4_F32 ? 1 : 0;

@@ -23,7 +23,7 @@ struct DebugReq {
 struct AttnArgs {
     int B, Hq, Hkv, N;
     int causal, out_dtype;
-    int head_major;               // CTA order: all query blocks of a head together (K/V larger than L2)
+    int group_heads;              // CTA order: groups of this many (batch, query head) pairs, one group after the other
     float c0, c1;                 // sigma, sigma * log2(e)
     int normalizer;               // 1: l accumulates the unquantized P (mismatched), not P-hat
     unsigned long long* hist;     // mass-error histogram [n_bins + 2] or null

@@ -142,12 +142,13 @@ attention_fwd_ws64_kernel(const __grid_constant__ CUtensorMap tmap_q, const __gr
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int N = args.N;
     const int n_qt = (N + 127) / 128;
-    // 1-D grid, query block outermost and descending: the heaviest causal CTAs are scheduled first
-    const int n_bh = args.B * args.Hq;
-    // Long sequences, whose K/V images do not fit in L2 together: head outermost instead, so that the
-    // CTAs in flight share the K/V of one or two heads; still heaviest first inside a head.
-    const int qt = n_qt - 1 - (int)(args.head_major ? blockIdx.x % n_qt : blockIdx.x / n_bh);
-    const int bh = (int)(args.head_major ? blockIdx.x / n_qt : blockIdx.x % n_bh);
+    // 1-D grid.  The (batch, query head) pairs are taken in groups whose K/V images fit in L2 together (one group
+    // when everything fits); inside a group the query block is outermost and descending, so that the heaviest
+    // causal CTAs are scheduled first and the CTAs in flight share the K/V of the group's heads.
+    const int gh = args.group_heads;                          // divides n_bh
+    const int grp_i = (int)blockIdx.x / (n_qt * gh), in_grp = (int)blockIdx.x % (n_qt * gh);
+    const int qt = n_qt - 1 - in_grp / gh;
+    const int bh = grp_i * gh + in_grp % gh;
     const int h = bh % args.Hq, b = bh / args.Hq;
     const int g = args.map.kv_of[h];
     const int q0 = qt * 128;
